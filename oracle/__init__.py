@@ -1,0 +1,21 @@
+"""CPU oracle for the PSO-PS synchronisation stage (test infrastructure).
+
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import
+this package.  It never imports the CUDA package and the CUDA package never
+imports it.
+"""
+from .psops_oracle import (  # noqa: F401
+    RefSwarm,
+    argmin,
+    average,
+    build,
+    draw,
+    inertia,
+    pbest_select,
+    philox4x32_10,
+    quadratic_fitness,
+    quadratic_losses,
+    sync,
+    uniform,
+    update_element,
+)
