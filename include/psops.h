@@ -1,0 +1,209 @@
+/*
+ * psops.h -- C ABI of the B200 PSO-PS parameter-synchronisation library.
+ *
+ * PSO-PS (Ye, Han, Sun, Lv, "PSO-PS: Parameter Synchronization with Particle
+ * Swarm Optimization for Distributed Training of Deep Neural Networks")
+ * replaces the averaging step of data-parallel training by a particle-swarm
+ * update: the K workers' weight vectors are particles (Table I: position =
+ * weights, fitness = training loss), each with a velocity and a personal best,
+ * and at every synchronisation point new weights come from Eq. 6 / Eq. 7
+ * instead of from the mean.  This library is that synchronisation stage for K
+ * particles held as K flat fp32 rows in one GPU's memory.
+ *
+ * Conventions
+ *   - All entry points return 0 (PSOPS_OK) or a negative PSOPS_E* code; none
+ *     throws, aborts or prints.  Arguments are validated before any launch.
+ *   - "device pointer" = address in the memory of the GPU that was current
+ *     when psops_create ran; "host pointer" = ordinary process memory.
+ *   - The library allocates no device memory.  The caller owns x, v, pbest,
+ *     the workspace, dvec/tvec and the stream, and keeps them alive until
+ *     psops_destroy.  The context itself is host memory owned by the library.
+ *   - Work is enqueued on the stream given at creation.  Calls that fill a
+ *     host buffer wait for that stream before they return; the others do not.
+ *   - Rows: particle i occupies elements [i*ld, i*ld + N) of x, v and pbest.
+ *     Elements [N, ld) of a row are padding and are never written.
+ *     If x, v, pbest are 16-byte aligned and ld % 4 == 0 the 128-bit kernels
+ *     run; otherwise a scalar variant with identical results runs.
+ *   - Random numbers: r1, r2 of Eq. 6 are drawn per (particle, element, sync)
+ *     from Philox4x32-10 with counter {element >> 1, particle, sync step, 0}
+ *     and key {seed low word, seed high word}; the even element of a pair
+ *     takes output words 0,1 and the odd element words 2,3; a word w becomes
+ *     (w >> 8) * 2^-24 in [0, 1).  The stream is a pure function of those
+ *     indices, so a context has no generator state beyond its step counter.
+ */
+#ifndef PSOPS_H
+#define PSOPS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PSOPS_OK           0
+#define PSOPS_EINVAL      -1   /* null pointer, size or hyper-parameter out of range   */
+#define PSOPS_EALIGN      -2   /* a device pointer is not 4-byte aligned               */
+#define PSOPS_ESTATE      -3   /* call order: e.g. sync before any losses were given   */
+#define PSOPS_ENAN        -4   /* a host-supplied loss is NaN                          */
+#define PSOPS_EWORKSPACE  -5   /* workspace missing, misaligned (256 B) or too small   */
+#define PSOPS_ECUDA       -6   /* a CUDA call failed; psops_last_error has its text    */
+#define PSOPS_ENOMEM      -7   /* host allocation of the context failed                */
+
+#define PSOPS_MAX_K     1024
+
+/* psops_config.flags */
+#define PSOPS_KEEP_GBEST   1u  /* keep a copy of the gBest row of each sync (+4N bytes of workspace) */
+#define PSOPS_QUADRATIC    2u  /* reserve workspace for the on-device quadratic fitness              */
+
+/* `which` of psops_get_weights / psops_set_weights */
+#define PSOPS_X      0         /* weights  w_i  (position of particle i)     */
+#define PSOPS_V      1         /* velocity v_i                               */
+#define PSOPS_PBEST  2         /* personal best pBest_i                      */
+#define PSOPS_GBEST  3         /* gBest of the last sync (needs KEEP_GBEST)  */
+
+typedef struct psops_ctx psops_ctx;      /* opaque */
+
+/* Hyper-parameters (Table II) and geometry of one swarm. */
+typedef struct {
+    int32_t  K;              /* particles = workers (Table I), 1..PSOPS_MAX_K              */
+    int64_t  N;              /* elements per particle, 1 .. 2^33 - 1                        */
+    int64_t  ld;             /* row stride in elements, ld >= N                             */
+    float    m_max, m_min;   /* Eq. 5; m_max == m_min gives a constant inertia weight       */
+    int64_t  t_max;          /* Eq. 5 denominator (Max_t of Algorithm 1), >= 1              */
+    float    c1, c2;         /* acceleration constants of Eq. 6                             */
+    uint64_t seed;           /* Philox key                                                  */
+    uint32_t flags;          /* PSOPS_KEEP_GBEST | PSOPS_QUADRATIC                          */
+} psops_config;
+
+/* Bytes of device workspace a context with this configuration needs
+ * (0 if the configuration is invalid).  The workspace must be 256-byte
+ * aligned. */
+size_t psops_workspace_bytes(const psops_config *cfg);
+
+/*
+ * Particle initialisation (Algorithm 2): adopt the caller's device rows as the
+ * swarm.  d_x, d_v, d_pbest: K rows of stride ld each, fp32, already holding
+ * the initial weights, velocities and personal bests (Algorithm 2 clones the
+ * weights, so callers normally pass pbest == a copy of x).  pBest_loss starts
+ * at +inf (the paper initialises no loss), the sync counter at 0.
+ * cuda_stream: a cudaStream_t (NULL = the legacy default stream).
+ * Errors: EINVAL, EALIGN, EWORKSPACE, ENOMEM, ECUDA.  On error *out is NULL.
+ */
+int psops_create(psops_ctx **out, const psops_config *cfg,
+                 float *d_x, float *d_v, float *d_pbest,
+                 void *d_workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Hand in the K current training losses (the fitness of Table I; lower is
+ * better).  on_device == 0: host pointer, checked for NaN (ENAN) and copied
+ * before the call returns to the stream (the buffer may be reused at once).
+ * on_device != 0: device pointer, copied on the stream, not inspected.
+ */
+int psops_set_losses(psops_ctx *ctx, const float *losses, int on_device);
+
+/*
+ * One synchronisation: the "t % step == 0" branch of Algorithm 1.
+ *   1. gBest = weights of the particle with the smallest loss at this
+ *      iteration (Algorithm 3); ties go to the lowest particle index; a NaN
+ *      loss never beats a number.
+ *   2. every particle with loss_i < pBest_loss_i (strict) sets pBest_i to its
+ *      current weights and pBest_loss_i to loss_i.
+ *   3. v_i <- m v_i + (c1 r1/lambda)(pBest_i - w_i) + (c2 r2/lambda)(gBest - w_i)
+ *      (Eq. 6) and w_i <- w_i + v_i (Eq. 7), with m from Eq. 5 at iteration
+ *      t_iter (clamped to t_max).  Rounding sequence per element, all fp32
+ *      round-to-nearest: dl = pBest - w; dg = gBest - w; t1 = (c1/lambda) r1;
+ *      t2 = (c2/lambda) r2; a0 = m v; v' = fma(t2, dg, fma(t1, dl, a0));
+ *      w' = w + v'.
+ * If a quadratic fitness is attached (psops_set_quadratic) the losses of the
+ * NEW weights are evaluated in the same pass and become the losses of the next
+ * sync.  Enqueues work only; the sync counter advances by one.
+ * Errors: EINVAL (t_iter < 0, lambda < 1 or not finite), ESTATE (no losses
+ * yet), ECUDA.
+ */
+int psops_sync(psops_ctx *ctx, int64_t t_iter, float lambda);
+
+/*
+ * Same synchronisation for callers whose weights live in host memory (the
+ * workers' side of Algorithm 1: gather weights and losses, distribute new
+ * weights).  h_x_in: K rows of stride h_in_ld (>= N) with the workers' current
+ * weights; h_losses: K losses; h_x_out: K rows of stride h_out_ld receiving
+ * the new weights (may equal h_x_in).  Velocities and personal bests stay on
+ * the device.  Copies and kernels are pipelined over element ranges; the call
+ * returns when h_x_out is complete.  Pinned host memory gives full speed.
+ * Errors: as psops_sync, plus ENAN.
+ */
+int psops_sync_host(psops_ctx *ctx, const float *h_x_in, int64_t h_in_ld,
+                    const float *h_losses, int64_t t_iter, float lambda,
+                    float *h_x_out, int64_t h_out_ld);
+
+/*
+ * Parameter averaging, the baseline the paper compares with (Section II-B,
+ * step 5): every w_i <- (1/K) sum_k w_k.  fp32 sum in particle order, one
+ * division.  Velocities, personal bests and the sync counter are untouched.
+ */
+int psops_average(psops_ctx *ctx);
+
+/*
+ * Copy one row out.  which = PSOPS_X / PSOPS_V / PSOPS_PBEST with particle k in
+ * [0, K), or PSOPS_GBEST (k ignored): the gBest row used by the last sync,
+ * available only with PSOPS_KEEP_GBEST (else ESTATE, as the pre-update row no
+ * longer exists).  dst receives N floats; dst_on_device selects the kind of
+ * pointer; a host destination is complete on return.
+ */
+int psops_get_weights(psops_ctx *ctx, int which, int k, float *dst, int dst_on_device);
+
+/* Overwrite row k of x, v or pbest with N floats from src (host or device). */
+int psops_set_weights(psops_ctx *ctx, int which, int k, const float *src, int src_on_device);
+
+/*
+ * Selection results of the last sync, copied to host memory (each pointer may
+ * be NULL): *g = gBest index; improved_words[(K+31)/32], bit i set when
+ * particle i improved; pbest_loss[K] after the update.  Waits for the stream.
+ * ESTATE before the first sync.
+ */
+int psops_sync_info(psops_ctx *ctx, int *g, uint32_t *improved_words, float *pbest_loss);
+
+/* The K losses currently held on the device, to dst (host or device). */
+int psops_get_losses(psops_ctx *ctx, float *dst, int dst_on_device);
+
+/*
+ * Attach the quadratic stand-in fitness f(w) = sum_j dvec_j (w_j - tvec_j)^2
+ * (device pointers, N floats each, borrowed; both NULL detaches).  Needs
+ * PSOPS_QUADRATIC.  The summation order is fixed so that results are
+ * reproducible bit for bit: fp32 terms dvec*(e*e) widened to fp64; four
+ * consecutive terms added left to right; 32 such sums (128 elements) combined
+ * by the butterfly a[l] += a[l ^ off], off = 16..1; tile sums added into 1024
+ * slots (tile m -> slot m % 1024, increasing m, from +0.0); slots combined as
+ * 32 butterflies of 32 and the 32 results added in order; rounded to fp32.
+ */
+int psops_set_quadratic(psops_ctx *ctx, const float *d_dvec, const float *d_tvec);
+
+/* losses <- f(current weights) for every particle (the evaluation that
+ * precedes the first sync). */
+int psops_eval_quadratic(psops_ctx *ctx);
+
+/* Checkpoint / resume of the small state: the sync counter and pBest_loss[K]
+ * (host pointers).  x, v, pbest are the caller's own tensors. */
+int psops_get_state(psops_ctx *ctx, uint32_t *sync_step, float *pbest_loss);
+int psops_set_state(psops_ctx *ctx, uint32_t sync_step, const float *pbest_loss);
+
+/* Inertia weight of Eq. 5 as psops_sync would compute it (host only). */
+float psops_inertia(const psops_config *cfg, int64_t t_iter);
+
+/* Number of kernel launches this context has enqueued so far. */
+int64_t psops_launch_count(const psops_ctx *ctx);
+
+/* Static description of an error code. */
+const char *psops_strerror(int code);
+
+/* Text of the last CUDA error seen by this context ("" if none). */
+const char *psops_last_error(const psops_ctx *ctx);
+
+/* Waits for the stream, then frees the context (not the caller's buffers). */
+int psops_destroy(psops_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PSOPS_H */

@@ -1,0 +1,476 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle on
+the same seeded inputs -- selection bit-exact, x / v / pbest within 1e-6
+relative after every sync, free-running (the GPU state is never refreshed from
+the oracle)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2009_03816_b200 import binding, workloads
+from paper_2009_03816_b200.binding import (PSOPS_GBEST, PSOPS_KEEP_GBEST, PSOPS_PBEST,
+                                           PSOPS_QUADRATIC, PSOPS_V, PSOPS_X)
+
+import gpu_util
+from gpu_util import NTHREADS, Pair, assert_close
+
+pytestmark = pytest.mark.gpu
+
+
+def _swarm(K, N, seed, sv=0.1):
+    rng = np.random.default_rng(seed)
+    x = rng.standard_normal((K, N)).astype(np.float32)
+    v = (sv * rng.standard_normal((K, N))).astype(np.float32)
+    p = (x + 0.5 * rng.standard_normal((K, N))).astype(np.float32)
+    return x, v, p
+
+
+# ---------------------------------------------------------------------------
+# Small shapes: several tiles, ragged tails, both kernels variants.
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("N", [1, 2, 3, 5, 127, 128, 129, 1000, 4099])
+@pytest.mark.parametrize("K", [1, 2, 3, 32, 33])
+def test_small_shapes_vector_path(K, N):
+    x, v, p = _swarm(K, N, 100 * K + N)
+    pair = Pair(x, v, p, N, m_max=0.9, m_min=0.3, t_max=10, c1=0.2, c2=0.9, seed=K * 7919 + N)
+    rng = np.random.default_rng(N)
+    for s in range(4):
+        pair.sync(rng.random(K).astype(np.float32), t=3 * s, lam=1.0 + s)
+        pair.check_selection()
+        pair.check_state(f"K={K} N={N} s={s}")
+    pair.check_canaries()
+    assert pair.inexact == 0          # same rounding sequence on both sides
+    pair.close()
+
+
+@pytest.mark.parametrize("N,ld,offset", [(5, 5, 0), (129, 131, 0), (1000, 1000, 1), (1003, 1003, 3),
+                                         (4096, 4096, 2), (777, 780, 1)])
+@pytest.mark.parametrize("K", [1, 4, 33])
+def test_small_shapes_scalar_path(K, N, ld, offset):
+    x, v, p = _swarm(K, N, 3 * K + N)
+    pair = Pair(x, v, p, N, ld=ld, offset=offset, m_max=0.7, m_min=0.7, c1=1.5, c2=1.5, seed=N)
+    rng = np.random.default_rng(K)
+    for s in range(3):
+        pair.sync(rng.random(K).astype(np.float32))
+        pair.check_selection()
+        pair.check_state(f"K={K} N={N} ld={ld} off={offset} s={s}")
+    pair.check_canaries()
+    assert pair.inexact == 0
+    pair.close()
+
+
+def test_many_particles():
+    K, N = binding.PSOPS_MAX_K, 260
+    x, v, p = _swarm(K, N, 5)
+    pair = Pair(x, v, p, N, m_max=0.7, m_min=0.7, c1=1.5, c2=1.5, seed=11)
+    rng = np.random.default_rng(2)
+    for s in range(3):
+        loss = rng.integers(0, 50, size=K).astype(np.float32)      # many ties
+        pair.sync(loss)
+        pair.check_selection()
+    pair.check_state("K=1024")
+    pair.check_canaries()
+    pair.close()
+
+
+# ---------------------------------------------------------------------------
+# Selection edge cases through the device kernel.
+# ---------------------------------------------------------------------------
+def test_selection_ties_nan_inf_on_device():
+    K, N = 40, 64
+    x, v, p = _swarm(K, N, 9)
+    pair = Pair(x, v, p, N, m_max=0.7, m_min=0.7, c1=1.5, c2=1.5, seed=3)
+    rng = np.random.default_rng(1)
+    cases = []
+    for _ in range(20):
+        loss = rng.integers(0, 3, size=K).astype(np.float32)
+        cases.append(loss)
+    cases.append(np.full(K, np.inf, np.float32))
+    cases.append(np.where(np.arange(K) == 37, -0.0, 0.0).astype(np.float32))
+    for loss in cases:
+        pair.sync(loss)
+        pair.check_selection()
+    # device-side NaN losses (the host path refuses them): they never win
+    dl = np.full(K, np.nan, np.float32)
+    dl[35] = 5.0
+    dl[36] = 5.0
+    dev = torch.from_numpy(dl).cuda()
+    pair.gpu.set_losses(dev)
+    pair.gpu.sync()
+    pair.ref.sync(dl)
+    pair.check_selection()
+    assert pair.ref.g == 35
+    dev = torch.from_numpy(np.full(K, np.nan, np.float32)).cuda()
+    pair.gpu.set_losses(dev)
+    pair.gpu.sync()
+    pair.ref.sync(np.full(K, np.nan, np.float32))
+    pair.check_selection()
+    assert pair.ref.g == 0
+    pair.close()
+
+
+@pytest.mark.parametrize("g", [0, 1, 2, 3, 4])
+def test_gbest_row_is_read_before_it_is_overwritten(g):
+    K, N = 5, 10_007
+    x, v, p = _swarm(K, N, 77)
+    pair = Pair(x, v, p, N, m_max=0.7, m_min=0.7, c1=1.5, c2=1.5, seed=g, flags=PSOPS_KEEP_GBEST)
+    loss = np.full(K, 2.0, np.float32)
+    loss[g] = 1.0
+    pair.sync(loss, want_gbest=True)
+    pair.check_selection()
+    assert pair.ref.g == g
+    pair.check_state(f"g={g}")
+    got = pair.gpu.row(PSOPS_GBEST)
+    assert np.array_equal(got, x[g]) and np.array_equal(got, pair.ref.gbest)
+    pair.close()
+
+
+# ---------------------------------------------------------------------------
+# The five workload recipes.
+# ---------------------------------------------------------------------------
+def _run_workload(w, every=1):
+    x, v, p = workloads.state(w)
+    table = workloads.losses(w)
+    pair = Pair(x, v, p, w.N, ld=w.ld, m_max=w.omega, m_min=w.omega, c1=w.c1, c2=w.c2, seed=w.seed)
+    for s in range(w.S):
+        pair.sync(table[s], 0, w.lam)
+        pair.check_selection()
+        if s % every == 0 or s == w.S - 1:
+            pair.check_state(f"{w.name} s={s}")
+    pair.check_canaries(w.name)
+    inexact = pair.inexact
+    pair.close()
+    return inexact
+
+
+def test_cfg1_full():
+    assert _run_workload(workloads.CONFIGS["cfg1"]) == 0
+
+
+def test_cfg2_full():
+    # omega=0.9, c=2.0 is outside PSO's stability region: trajectories amplify
+    # any rounding difference, so this only passes with identical rounding.
+    assert _run_workload(workloads.CONFIGS["cfg2"], every=7) == 0
+
+
+def test_cfg3_scaled_with_ties():
+    w = workloads.CONFIGS["cfg3"].scaled(N=300_002)
+    assert w.ld == 300_004
+    assert _run_workload(w, every=9) == 0
+
+
+def test_cfg4_scaled():
+    assert _run_workload(workloads.CONFIGS["cfg4"].scaled(N=131_072 + 40, S=30), every=5) == 0
+
+
+def _run_sampled(w, count):
+    """Full-size run on the GPU; the oracle follows a sample of columns (every
+    element is independent of the others once the losses are given)."""
+    gpu_util.ensure_library()
+    cols = workloads.sample_columns(w.N, count, w.seed)
+    dev = torch.device("cuda:0")
+    dx = torch.zeros((w.K, w.ld), dtype=torch.float32, device=dev)
+    dv = torch.zeros((w.K, w.ld), dtype=torch.float32, device=dev)
+    xs = np.empty((w.K, cols.size), np.float32)
+    vs = np.empty((w.K, cols.size), np.float32)
+    for k in range(w.K):
+        row = workloads.x_row(w, k)
+        xs[k] = row[cols]
+        dx[k, :w.N] = torch.from_numpy(row).to(dev)
+        row = workloads.v_row(w, k)
+        vs[k] = row[cols]
+        dv[k, :w.N] = torch.from_numpy(row).to(dev)
+    dp = dx.clone()
+    table = workloads.losses(w)
+    gpu = binding.Swarm(dx, dv, dp, N=w.N, m_max=w.omega, m_min=w.omega, c1=w.c1, c2=w.c2, seed=w.seed)
+    ref = oracle.RefSwarm(xs, vs, xs, m_max=w.omega, m_min=w.omega, t_max=1, c1=w.c1, c2=w.c2,
+                          seed=w.seed, elem_index=cols)
+    dtable = torch.from_numpy(table).to(dev)
+    dcols = torch.from_numpy(cols).to(dev)
+    inexact = 0
+    for s in range(w.S):
+        gpu.set_losses(dtable[s])                 # device-resident losses, as the benchmark does
+        gpu.sync(0, w.lam)
+        ref.sync(table[s], 0, w.lam)
+        g, improved, pl = gpu.info()
+        assert g == ref.g and np.array_equal(improved, ref.improved)
+        assert np.array_equal(pl.view(np.uint32), ref.pbest_loss.view(np.uint32))
+        if s % 10 == 0 or s == w.S - 1:
+            for name, t, want in (("x", dx, ref.x), ("v", dv, ref.v), ("pbest", dp, ref.p)):
+                got = t[:, dcols].cpu().numpy()
+                inexact += assert_close(got, want, f"{w.name} s={s} {name}")
+    assert torch.all(dx[:, w.N:] == 0) and torch.all(dv[:, w.N:] == 0) and torch.all(dp[:, w.N:] == 0)
+    gpu.close()
+    return inexact
+
+
+def test_cfg3_full_size_sampled():
+    assert _run_sampled(workloads.CONFIGS["cfg3"], 4000) == 0
+
+
+def test_cfg4_full_size_sampled():
+    assert _run_sampled(workloads.CONFIGS["cfg4"], 2000) == 0
+
+
+# ---------------------------------------------------------------------------
+# Quadratic fitness on the device (stand-alone and fused into the update).
+# ---------------------------------------------------------------------------
+def _quadratic_pair(w, flags=PSOPS_QUADRATIC):
+    x, v, p = workloads.state(w)
+    d, t = workloads.quadratic_vectors(w)
+    pair = Pair(x, v, p, w.N, ld=w.ld, m_max=w.omega, m_min=w.omega, c1=w.c1, c2=w.c2, seed=w.seed,
+                flags=flags)
+    dd, dt = torch.from_numpy(d).cuda(), torch.from_numpy(t).cuda()
+    pair.gpu.set_quadratic(dd, dt)
+    return pair, d, t
+
+
+@pytest.mark.parametrize("N", [1, 3, 127, 128, 129, 4096 + 5, 131_072 * 3 + 77])
+def test_quadratic_fitness_standalone_bit_exact(N):
+    w = workloads.CONFIGS["cfg5"].scaled(N=N)
+    pair, d, t = _quadratic_pair(w)
+    pair.gpu.eval_quadratic()
+    got = pair.gpu.losses()
+    want = oracle.quadratic_losses(pair.ref.x, d, t, nthreads=NTHREADS)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+    pair.close()
+
+
+def test_cfg5_scaled_fused_fitness_every_step():
+    w = workloads.CONFIGS["cfg5"].scaled(N=1_000_003, S=200)
+    pair, d, t = _quadratic_pair(w)
+    pair.gpu.eval_quadratic()
+    loss = oracle.quadratic_losses(pair.ref.x, d, t, nthreads=NTHREADS)
+    best = []
+    for s in range(w.S):
+        assert np.array_equal(pair.gpu.losses().view(np.uint32), loss.view(np.uint32)), s
+        pair.gpu.sync(0, w.lam)                   # losses come from the device
+        pair.ref.sync(loss, 0, w.lam)
+        pair.check_selection()
+        loss = oracle.quadratic_losses(pair.ref.x, d, t, nthreads=NTHREADS)
+        if s % 20 == 0 or s == w.S - 1:
+            pair.check_state(f"{w.name} s={s}")
+        best.append(float(pair.ref.pbest_loss.min()))
+    assert np.array_equal(pair.gpu.losses().view(np.uint32), loss.view(np.uint32))
+    assert all(a >= b for a, b in zip(best, best[1:]))
+    assert pair.inexact == 0
+    pair.check_canaries()
+    pair.close()
+
+
+def test_cfg5_scalar_path_fused_fitness():
+    w = workloads.CONFIGS["cfg5"].scaled(N=70_001, S=5)
+    x, v, p = workloads.state(w)
+    d, t = workloads.quadratic_vectors(w)
+    pair = Pair(x, v, p, w.N, ld=w.N, offset=1, m_max=w.omega, m_min=w.omega, c1=w.c1, c2=w.c2,
+                seed=w.seed, flags=PSOPS_QUADRATIC)
+    dd, dt = torch.from_numpy(d).cuda(), torch.from_numpy(t).cuda()
+    pair.gpu.set_quadratic(dd, dt)
+    pair.gpu.eval_quadratic()
+    loss = oracle.quadratic_losses(pair.ref.x, d, t)
+    for s in range(w.S):
+        assert np.array_equal(pair.gpu.losses().view(np.uint32), loss.view(np.uint32))
+        pair.gpu.sync()
+        pair.ref.sync(loss)
+        pair.check_selection()
+        pair.check_state(f"s={s}")
+        loss = oracle.quadratic_losses(pair.ref.x, d, t)
+    pair.check_canaries()
+    pair.close()
+
+
+def test_cfg5_full_size_two_syncs():
+    """Full 50 M-element vectors, fitness fused into the update; the oracle
+    runs the whole swarm on all host cores for a bounded number of syncs."""
+    w = workloads.CONFIGS["cfg5"]
+    gpu_util.ensure_library()
+    dev = torch.device("cuda:0")
+    x, v, p = workloads.state(w)
+    d, t = workloads.quadratic_vectors(w)
+    dx, dv = torch.from_numpy(x).to(dev), torch.from_numpy(v).to(dev)
+    dp = dx.clone()
+    dd, dt = torch.from_numpy(d).to(dev), torch.from_numpy(t).to(dev)
+    gpu = binding.Swarm(dx, dv, dp, N=w.N, m_max=w.omega, m_min=w.omega, c1=w.c1, c2=w.c2,
+                        seed=w.seed, flags=PSOPS_QUADRATIC)
+    gpu.set_quadratic(dd, dt)
+    gpu.eval_quadratic()
+    ref = oracle.RefSwarm(x, v, p, m_max=w.omega, m_min=w.omega, t_max=1, c1=w.c1, c2=w.c2,
+                          seed=w.seed, nthreads=NTHREADS)
+    del x, v, p
+    loss = oracle.quadratic_losses(ref.x, d, t, nthreads=NTHREADS)
+    cols = torch.from_numpy(workloads.sample_columns(w.N, 200_000, 5)).to(dev)
+    for s in range(2):
+        assert np.array_equal(gpu.losses().view(np.uint32), loss.view(np.uint32))
+        gpu.sync(0, w.lam)
+        ref.sync(loss, 0, w.lam)
+        g, improved, pl = gpu.info()
+        assert g == ref.g and np.array_equal(improved, ref.improved)
+        loss = oracle.quadratic_losses(ref.x, d, t, nthreads=NTHREADS)
+    assert np.array_equal(gpu.losses().view(np.uint32), loss.view(np.uint32))
+    hc = cols.cpu().numpy()
+    for name, tdev, want in (("x", dx, ref.x), ("v", dv, ref.v), ("pbest", dp, ref.p)):
+        assert assert_close(tdev[:, cols].cpu().numpy(), want[:, hc], name) == 0
+    gpu.close()
+
+
+# ---------------------------------------------------------------------------
+# Parameter averaging.
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("K,N,ld,offset", [(1, 100, 100, 0), (2, 1001, 1004, 0), (16, 300_002, 300_004, 0),
+                                           (7, 999, 999, 1), (32, 70_000, 70_000, 0), (33, 5, 8, 0)])
+def test_average_bit_exact(K, N, ld, offset):
+    x, v, p = _swarm(K, N, K + N)
+    pair = Pair(x, v, p, N, ld=ld, offset=offset, m_max=0.7, m_min=0.7, c1=1.5, c2=1.5, seed=1)
+    pair.gpu.average()
+    pair.ref.average()
+    got = pair.dx.host()
+    assert np.array_equal(got.view(np.uint32), pair.ref.x.view(np.uint32))
+    assert np.array_equal(pair.dv.host(), v) and np.array_equal(pair.dp.host(), p)   # untouched
+    pair.check_canaries()
+    # averaging then a sync still follows the oracle
+    pair.sync(np.linspace(1, 2, K).astype(np.float32))
+    pair.check_selection()
+    pair.check_state("after average")
+    pair.close()
+
+
+# ---------------------------------------------------------------------------
+# Host-buffer entry point, row access, determinism, resume.
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("pinned", [False, True])
+def test_sync_host_matches_oracle(pinned):
+    w = workloads.CONFIGS["cfg2"].scaled(N=2_500_001, S=3)     # several pipeline ranges + ragged tail
+    x, v, p = workloads.state(w)
+    table = workloads.losses(w)
+    pair = Pair(x, v, p, w.N, ld=w.ld, m_max=w.omega, m_min=w.omega, c1=w.c1, c2=w.c2, seed=w.seed)
+    h_in = torch.from_numpy(x.copy())
+    h_out = torch.full((w.K, w.ld), 123.0)
+    if pinned:
+        h_in, h_out = h_in.pin_memory(), h_out.pin_memory()
+    for s in range(w.S):
+        # the workers' weights arrive from the host each time
+        h_in[:, :w.N] = torch.from_numpy(pair.ref.x)
+        pair.gpu.sync_host(h_in, table[s], 0, w.lam, h_out)
+        pair.ref.sync(table[s], 0, w.lam)
+        pair.check_selection()
+        assert assert_close(h_out.numpy()[:, :w.N], pair.ref.x, "host out") == 0
+        assert torch.all(h_out[:, w.N:] == 123.0)
+        pair.check_state(f"sync_host s={s}")
+    pair.check_canaries()
+    pair.close()
+
+
+def test_get_and_set_weights_rows():
+    K, N = 3, 1001
+    x, v, p = _swarm(K, N, 1)
+    pair = Pair(x, v, p, N, m_max=0.7, m_min=0.7, c1=1.5, c2=1.5, seed=1)
+    for which, src in ((PSOPS_X, x), (PSOPS_V, v), (PSOPS_PBEST, p)):
+        for k in range(K):
+            assert np.array_equal(pair.gpu.row(which, k), src[k])
+    new = np.arange(N, dtype=np.float32)
+    binding.psops_set_weights(pair.gpu.ctx, PSOPS_V, 1, new)
+    assert np.array_equal(pair.gpu.row(PSOPS_V, 1), new)
+    dev_dst = torch.empty(N, device="cuda")
+    binding.psops_get_weights(pair.gpu.ctx, PSOPS_X, 2, dev_dst)
+    assert np.array_equal(dev_dst.cpu().numpy(), x[2])
+    with pytest.raises(binding.PsopsError) as e:
+        pair.gpu.row(PSOPS_GBEST)
+    assert e.value.code == binding.PSOPS_ESTATE
+    with pytest.raises(binding.PsopsError):
+        pair.gpu.row(PSOPS_X, K)
+    pair.check_canaries()
+    pair.close()
+
+
+def test_deterministic_and_resumable():
+    w = workloads.CONFIGS["cfg1"].scaled(N=50_001, S=10)
+    x, v, p = workloads.state(w)
+    table = workloads.losses(w)
+    kw = dict(N=w.N, m_max=w.omega, m_min=w.omega, c1=w.c1, c2=w.c2, seed=w.seed)
+
+    def fresh():
+        return [torch.from_numpy(a).cuda() for a in (x, v, p)]
+
+    a = fresh()
+    sa = binding.Swarm(*a, **kw)
+    for s in range(10):
+        sa.set_losses(table[s])
+        sa.sync()
+    b = fresh()
+    sb = binding.Swarm(*b, **kw)
+    for s in range(5):
+        sb.set_losses(table[s])
+        sb.sync()
+    step, pl = sb.state()
+    assert step == 5
+    sb.close()
+    sc = binding.Swarm(*b, **kw)          # new context on the same tensors
+    sc.set_state(step, pl)
+    for s in range(5, 10):
+        sc.set_losses(table[s])
+        sc.sync()
+    torch.cuda.synchronize()
+    for ta, tb in zip(a, b):
+        assert torch.equal(ta, tb)
+    assert sa.info()[0] == sc.info()[0] and np.array_equal(sa.info()[2], sc.info()[2])
+    sa.close()
+    sc.close()
+
+
+def test_runs_on_a_side_stream_and_counts_launches():
+    K, N = 4, 20_000
+    x, v, p = _swarm(K, N, 4)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        t = [torch.from_numpy(a).cuda() for a in (x, v, p)]
+    stream.synchronize()
+    sw = binding.Swarm(*t, N=N, m_max=0.7, m_min=0.7, c1=1.5, c2=1.5, seed=8, stream=stream.cuda_stream)
+    ref = oracle.RefSwarm(x, v, p, m_max=0.7, m_min=0.7, t_max=1, c1=1.5, c2=1.5, seed=8)
+    loss = np.array([4, 3, 2, 1], np.float32)
+    sw.set_losses(loss)
+    sw.sync()
+    ref.sync(loss)
+    stream.synchronize()
+    assert sw.launches == 2                        # selection + fused update
+    assert assert_close(t[0].cpu().numpy(), ref.x) == 0
+    sw.average()
+    assert sw.launches == 3
+    sw.close()
+
+
+def test_device_errors_and_call_order():
+    K, N = 2, 64
+    x, v, p = _swarm(K, N, 4)
+    t = [torch.from_numpy(a).cuda() for a in (x, v, p)]
+    sw = binding.Swarm(*t, N=N, m_max=0.7, m_min=0.7, c1=1.5, c2=1.5, seed=8)
+    before = [a.clone() for a in t]
+    codes = []
+    for fn in (lambda: sw.sync(),                                   # no losses yet
+               lambda: sw.set_losses(np.array([np.nan, 1.0], np.float32)),
+               lambda: sw.info(),
+               lambda: sw.eval_quadratic(),
+               lambda: sw.set_quadratic(t[0], t[1])):               # no QUADRATIC workspace
+        with pytest.raises(binding.PsopsError) as e:
+            fn()
+        codes.append(e.value.code)
+    assert codes == [binding.PSOPS_ESTATE, binding.PSOPS_ENAN, binding.PSOPS_ESTATE,
+                     binding.PSOPS_ESTATE, binding.PSOPS_EWORKSPACE]
+    sw.set_losses([1.0, 2.0])
+    for bad in (lambda: sw.sync(-1, 1.0), lambda: sw.sync(0, 0.5), lambda: sw.sync(0, float("nan")),
+                lambda: sw.sync(0, float("inf"))):
+        with pytest.raises(binding.PsopsError) as e:
+            bad()
+        assert e.value.code == binding.PSOPS_EINVAL
+    torch.cuda.synchronize()
+    assert all(torch.equal(a, b) for a, b in zip(t, before))        # nothing was touched
+    assert sw.launches == 0
+    # misaligned or undersized workspace
+    cfg = sw.cfg
+    ws = torch.empty(binding.psops_workspace_bytes(cfg) + 512, dtype=torch.uint8, device="cuda")
+    with pytest.raises(binding.PsopsError) as e:
+        binding.psops_create(cfg, *t, ws[4:], ws.numel() - 4)
+    assert e.value.code == binding.PSOPS_EWORKSPACE
+    with pytest.raises(binding.PsopsError) as e:
+        binding.psops_create(cfg, *t, ws, 16)
+    assert e.value.code == binding.PSOPS_EWORKSPACE
+    sw.close()
