@@ -49,6 +49,7 @@ extern "C" {
 #define PSOPS_EWORKSPACE  -5   /* workspace missing, misaligned (256 B) or too small   */
 #define PSOPS_ECUDA       -6   /* a CUDA call failed; psops_last_error has its text    */
 #define PSOPS_ENOMEM      -7   /* host allocation of the context failed                */
+#define PSOPS_ELIMIT      -8   /* size beyond the built-in scratch (psops_quadratic_fitness_static) */
 
 #define PSOPS_MAX_K     1024
 
@@ -182,6 +183,38 @@ int psops_set_quadratic(psops_ctx *ctx, const float *d_dvec, const float *d_tvec
 /* losses <- f(current weights) for every particle (the evaluation that
  * precedes the first sync). */
 int psops_eval_quadratic(psops_ctx *ctx);
+
+/*
+ * (No counterpart in the paper: an addition for callers that cannot allocate.)
+ * The quadratic fitness of K rows without any workspace and without a context:
+ * d_loss[i] = f(row i of d_x), the same value, bit for bit, that
+ * psops_eval_quadratic produces.  It is meant for code that has no way to get
+ * device memory when it needs the value: inside a loop whose framework already
+ * owns all of the GPU's memory through its caching allocator, in a plug-in that
+ * is handed nothing but input and output buffers, or where cudaMalloc/cudaFree
+ * are off limits because they stall every stream of the device.  The call
+ * itself allocates nothing, on the host or on the device.
+ *   d_x            K rows of stride ld (>= N) fp32, device pointer
+ *   d_dvec, d_tvec N fp32 each, device pointers
+ *   d_loss         K fp32, device pointer, written on the stream
+ *   cuda_stream    a cudaStream_t (NULL = legacy default stream); work is only
+ *                  enqueued
+ * The intermediate tile sums go to an array of PSOPS_STATIC_SCRATCH_DOUBLES
+ * doubles (8 MiB) that is built into the library and therefore occupies that
+ * much memory on every GPU that loads it until the process exits.  A problem
+ * with K * ceil(N/128) above that number is refused with PSOPS_ELIMIT and
+ * nothing is launched.  The first call on each device looks the array's address
+ * up (the device must be current) -- make that first call outside any stream
+ * capture.  All calls on a device share the array and it is not cleared
+ * between calls (every slot that is read has been written by the same call);
+ * calls that overlap in time on one GPU overwrite each other's partial results,
+ * so keep them on one stream or order them yourself.
+ * Errors: EINVAL, EALIGN (a pointer not 4-byte aligned), ELIMIT, ECUDA.
+ */
+#define PSOPS_STATIC_SCRATCH_DOUBLES (1 << 20)
+int psops_quadratic_fitness_static(const float *d_x, int64_t ld, int32_t K, int64_t N,
+                                   const float *d_dvec, const float *d_tvec,
+                                   float *d_loss, void *cuda_stream);
 
 /* Checkpoint / resume of the small state: the sync counter and pBest_loss[K]
  * (host pointers).  x, v, pbest are the caller's own tensors. */

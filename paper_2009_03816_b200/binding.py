@@ -18,7 +18,8 @@ from .build import LIBRARY
 
 PSOPS_OK = 0
 PSOPS_EINVAL, PSOPS_EALIGN, PSOPS_ESTATE, PSOPS_ENAN = -1, -2, -3, -4
-PSOPS_EWORKSPACE, PSOPS_ECUDA, PSOPS_ENOMEM = -5, -6, -7
+PSOPS_EWORKSPACE, PSOPS_ECUDA, PSOPS_ENOMEM, PSOPS_ELIMIT = -5, -6, -7, -8
+PSOPS_STATIC_SCRATCH_DOUBLES = 1 << 20
 PSOPS_MAX_K = 1024
 PSOPS_KEEP_GBEST, PSOPS_QUADRATIC = 1, 2
 PSOPS_X, PSOPS_V, PSOPS_PBEST, PSOPS_GBEST = 0, 1, 2, 3
@@ -29,6 +30,7 @@ EXPORTS = [
     "psops_sync_info", "psops_get_losses", "psops_set_quadratic",
     "psops_eval_quadratic", "psops_get_state", "psops_set_state", "psops_inertia",
     "psops_launch_count", "psops_strerror", "psops_last_error", "psops_destroy",
+    "psops_quadratic_fitness_static",
 ]
 
 
@@ -86,6 +88,8 @@ def load() -> ctypes.CDLL:
         "psops_strerror": (ctypes.c_char_p, [ctypes.c_int]),
         "psops_last_error": (ctypes.c_char_p, [_vp]),
         "psops_destroy": (ctypes.c_int, [_vp]),
+        "psops_quadratic_fitness_static": (ctypes.c_int, [_f32p, ctypes.c_int64, ctypes.c_int32,
+                                                          ctypes.c_int64, _f32p, _f32p, _f32p, _vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)            # AttributeError if a symbol is missing
@@ -219,6 +223,16 @@ def psops_launch_count(ctx) -> int:
 
 def psops_destroy(ctx) -> None:
     _check(load().psops_destroy(ctx), "psops_destroy")
+
+
+def psops_quadratic_fitness_static(d_x, ld, K, N, d_dvec, d_tvec, d_loss, stream=None) -> None:
+    """Fitness of K device rows into d_loss[K] using the library's built-in
+    scratch array: no workspace, no context, no allocation (for callers that
+    cannot allocate device memory).  Work is enqueued on `stream`."""
+    _check(load().psops_quadratic_fitness_static(_ptr(d_x), int(ld), int(K), int(N), _ptr(d_dvec),
+                                                 _ptr(d_tvec), _ptr(d_loss),
+                                                 int(stream) if stream else None),
+           "psops_quadratic_fitness_static")
 
 
 # ---- convenience holder of the tensors a context borrows ------------------

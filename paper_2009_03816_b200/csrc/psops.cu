@@ -23,6 +23,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -921,6 +922,7 @@ const char *psops_strerror(int code)
     case PSOPS_EWORKSPACE: return "workspace missing, misaligned or too small";
     case PSOPS_ECUDA: return "CUDA call failed";
     case PSOPS_ENOMEM: return "host allocation failed";
+    case PSOPS_ELIMIT: return "problem larger than the library's built-in scratch array";
     default: return "unknown error code";
     }
 }
@@ -940,3 +942,85 @@ int psops_destroy(psops_ctx *ctx)
 }
 
 } // extern "C"
+
+// ---------------------------------------------------------------------------
+// Allocation-free fitness evaluation.
+//
+// Some callers cannot obtain device memory at the moment they need a fitness
+// value: code running inside a serving or training loop whose framework has
+// already handed every byte of the GPU to its own caching allocator, plug-ins
+// that are only given input and output buffers, and latency-critical loops
+// that must not call cudaMalloc / cudaFree because those calls synchronise the
+// whole device.  For them the tile sums of the quadratic fitness live in a
+// fixed array that is part of this library's device image instead of in a
+// caller-provided workspace.
+//
+// The array costs PSOPS_STATIC_SCRATCH_DOUBLES * 8 bytes (8 MiB) on every GPU
+// that loads the library, for the life of the process.  All calls on a device
+// share it and it keeps whatever the previous call left there; the finaliser
+// reads only slots that the tile kernel of the same call has just written, so
+// nothing needs clearing.  Two calls that run concurrently on one GPU (two
+// streams, two host threads) would overwrite each other's tile sums.
+// ---------------------------------------------------------------------------
+static __device__ __align__(256) double psops_static_tile_sums[PSOPS_STATIC_SCRATCH_DOUBLES];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+double *g_static_tile_sums[kMaxDevices];      // device address of the array, per device ordinal
+bool g_static_ready[kMaxDevices];
+std::mutex g_static_mutex;
+
+// `psops_static_tile_sums` in host code is only a handle for the runtime, not
+// an address a kernel can use: resolve it once per device, with that device
+// current, and hand the result to the kernels.
+int static_scratch_for_current_device(double **ptr)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return PSOPS_ECUDA;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ready[dev]) {
+        void *addr = nullptr;
+        if (cudaGetSymbolAddress(&addr, psops_static_tile_sums) != cudaSuccess || addr == nullptr) {
+            (void)cudaGetLastError();
+            return PSOPS_ECUDA;
+        }
+        g_static_tile_sums[dev] = static_cast<double *>(addr);
+        g_static_ready[dev] = true;
+    }
+    *ptr = g_static_tile_sums[dev];
+    return PSOPS_OK;
+}
+
+} // namespace
+
+extern "C" int psops_quadratic_fitness_static(const float *d_x, int64_t ld, int32_t K, int64_t N,
+                                              const float *d_dvec, const float *d_tvec,
+                                              float *d_loss, void *cuda_stream)
+{
+    if (d_x == nullptr || d_dvec == nullptr || d_tvec == nullptr || d_loss == nullptr) return PSOPS_EINVAL;
+    if (K < 1 || K > PSOPS_MAX_K || N < 1 || N >= (1ll << 33) || ld < N) return PSOPS_EINVAL;
+    const uintptr_t bits = (uintptr_t)d_x | (uintptr_t)d_dvec | (uintptr_t)d_tvec;
+    if ((bits & 3u) || ((uintptr_t)d_loss & 3u)) return PSOPS_EALIGN;
+    const long long tiles = (N + kTileElems - 1) / kTileElems;
+    if ((long long)K * tiles > (long long)PSOPS_STATIC_SCRATCH_DOUBLES) return PSOPS_ELIMIT;
+
+    double *tile_sums = nullptr;
+    const int rc = static_scratch_for_current_device(&tile_sums);
+    if (rc != PSOPS_OK) return rc;
+
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const long long quads = (N + 3) / 4;
+    const unsigned blocks = (unsigned)((tiles * 32 + kUpdateThreads - 1) / kUpdateThreads);
+    const bool aligned = ((bits & 15u) == 0) && (ld % 4 == 0);
+    if (aligned)
+        psops_fitness_tiles_kernel<true><<<blocks, kUpdateThreads, 0, stream>>>(
+            d_x, d_dvec, d_tvec, tile_sums, ld, N, quads, tiles, K);
+    else
+        psops_fitness_tiles_kernel<false><<<blocks, kUpdateThreads, 0, stream>>>(
+            d_x, d_dvec, d_tvec, tile_sums, ld, N, quads, tiles, K);
+    if (cudaGetLastError() != cudaSuccess) return PSOPS_ECUDA;
+    psops_fitness_finalize_kernel<<<K, kFinalizeThreads, 0, stream>>>(tile_sums, d_loss, tiles);
+    if (cudaGetLastError() != cudaSuccess) return PSOPS_ECUDA;
+    return PSOPS_OK;
+}

@@ -84,9 +84,21 @@ def test_create_rejects_bad_arguments_before_touching_cuda(lib):
     assert lib.psops_launch_count(null) == 0
 
 
+def test_static_fitness_validates_before_touching_cuda(lib):
+    fake = 0x10000                                                    # never dereferenced
+    f = lib.psops_quadratic_fitness_static
+    assert f(None, 100, 2, 100, fake, fake, fake, None) == binding.PSOPS_EINVAL
+    assert f(fake, 100, 2, 100, fake, fake, None, None) == binding.PSOPS_EINVAL
+    assert f(fake, 99, 2, 100, fake, fake, fake, None) == binding.PSOPS_EINVAL      # ld < N
+    assert f(fake, 100, 0, 100, fake, fake, fake, None) == binding.PSOPS_EINVAL
+    assert f(fake + 1, 100, 2, 100, fake, fake, fake, None) == binding.PSOPS_EALIGN
+    n = 128 * binding.PSOPS_STATIC_SCRATCH_DOUBLES
+    assert f(fake, n, 2, n, fake, fake, fake, None) == binding.PSOPS_ELIMIT         # 2 * tiles > limit
+
+
 def test_strerror_is_distinct_per_code(lib):
-    texts = {lib.psops_strerror(c).decode() for c in range(0, -8, -1)}
-    assert len(texts) == 8
+    texts = {lib.psops_strerror(c).decode() for c in range(0, -9, -1)}
+    assert len(texts) == 9
     assert lib.psops_strerror(-99).decode() == "unknown error code"
 
 
