@@ -43,7 +43,9 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["psops", "reference"], default="psops")
     ap.add_argument("--workload", default="cfg4")
-    ap.add_argument("--e2e-steps", type=int, default=4)
+    ap.add_argument("--n", type=int, default=0,
+                    help="run the workload's recipe at this vector length instead (profiling captures)")
+    ap.add_argument("--e2e-steps", type=int, default=4, help="0 skips the host-buffer measurement")
     ap.add_argument("--rows", choices=["all", "none"], default="all",
                     help="also time the other rows of the path (averaging, cfg3, fused fitness)")
     ap.add_argument("--cpu-baseline", choices=["on", "off"], default="on")
@@ -237,6 +239,8 @@ def run_psops(args):
     torch.cuda.set_device(ranks.local_rank)
     dev = torch.device("cuda", ranks.local_rank)
     w = workloads.CONFIGS[args.workload]
+    if args.n:
+        w = w.scaled(N=args.n)
     peak, peak_src = measured_peak()
     pe = w.K * w.N
 
@@ -248,25 +252,31 @@ def run_psops(args):
     achieved = sync_bytes(w, fused) / (seconds / args.steps) / 1e9
 
     # ---- end to end: host buffers in, host buffers out, through psops_sync_host
-    table = workloads.losses(w) if not fused else None
-    h_in = torch.empty((w.K, w.ld), dtype=torch.float32).pin_memory()
-    h_out = torch.empty((w.K, w.ld), dtype=torch.float32).pin_memory()
-    h_in.copy_(sw.x)
-    hl = np.ascontiguousarray(table[0]) if table is not None else sw.losses()
+    e2e = None
+    if args.e2e_steps > 0:
+        table = workloads.losses(w) if not fused else None
+        h_in = torch.empty((w.K, w.ld), dtype=torch.float32).pin_memory()
+        h_out = torch.empty((w.K, w.ld), dtype=torch.float32).pin_memory()
+        h_in.copy_(sw.x)
+        hl = np.ascontiguousarray(table[0]) if table is not None else sw.losses()
 
-    def e2e_step(i):
-        sw.sync_host(h_in, hl if table is None else table[i % table.shape[0]], 0, w.lam, h_out)
+        def e2e_step(i):
+            sw.sync_host(h_in, hl if table is None else table[i % table.shape[0]], 0, w.lam, h_out)
 
-    e2e_step(0)
-    torch.cuda.synchronize()
-    replicas.barrier(ranks)
-    t0 = time.perf_counter()
-    for i in range(args.e2e_steps):
-        e2e_step(1 + i)
-    torch.cuda.synchronize()
-    e2e_seconds = time.perf_counter() - t0
-    e2e_rate, _ = replicas.whole_job_rate(ranks, pe * args.e2e_steps, e2e_seconds)
-    del h_in, h_out
+        e2e_step(0)
+        torch.cuda.synchronize()
+        replicas.barrier(ranks)
+        t0 = time.perf_counter()
+        for i in range(args.e2e_steps):
+            e2e_step(1 + i)
+        torch.cuda.synchronize()
+        e2e_seconds = time.perf_counter() - t0
+        e2e_rate, _ = replicas.whole_job_rate(ranks, pe * args.e2e_steps, e2e_seconds)
+        del h_in, h_out
+        e2e = {"value": e2e_rate, "unit": UNIT, "h2d_bytes_per_step": 4 * w.K * w.N + 4 * w.K,
+               "d2h_bytes_per_step": 4 * w.K * w.N, "steps": args.e2e_steps,
+               "ms_per_step": e2e_seconds * 1e3 / args.e2e_steps,
+               "call": "psops_sync_host (pinned host weights in, new weights out)"}
 
     out = {
         "metric": METRIC, "value": rate, "unit": UNIT, "n_gpus": ranks.world,
@@ -279,10 +289,7 @@ def run_psops(args):
                    "l2": "state (12*K*N bytes) exceeds L2; no flush needed",
                    "parallelism": "replicas only"},
         "clocks": sampler.report(),
-        "e2e": {"value": e2e_rate, "unit": UNIT, "h2d_bytes_per_step": 4 * w.K * w.N + 4 * w.K,
-                "d2h_bytes_per_step": 4 * w.K * w.N, "steps": args.e2e_steps,
-                "ms_per_step": e2e_seconds * 1e3 / args.e2e_steps,
-                "call": "psops_sync_host (pinned host weights in, new weights out)"},
+        "e2e": e2e,
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "kernel": "psops_update_kernel", "achieved": achieved,
                      "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
