@@ -33,7 +33,9 @@ FALLBACK_HBM_GBS = 6650.0           # earlier measurement on this machine, used onl
 # DRAM traffic of the fused update kernel from an ncu capture, per
 # particle-element, and the hash of the kernel source it was taken from.  The
 # benchmark reports null once the source has changed.
-NCU_TRAFFIC = {"source_sha256": None, "bytes_per_particle_element": None, "profile": None}
+NCU_TRAFFIC = {"source_sha256": "73b09bcfd014706686406a4faf043dd5d0d70b5a9c9fffe5a1277ea33e69777e",
+               "bytes_per_particle_element": 19.56,       # 2.503 GB / 128 M at K=32, N=4 M
+               "profile": "profiles/update_kernel_cfg4_n4m_full.txt"}
 
 
 def parse_args():
