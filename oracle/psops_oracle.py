@@ -46,7 +46,9 @@ def _load():
     with _lock:
         if _lib is not None:
             return _lib
-        lib = ctypes.CDLL(build())
+        # PSOPS_REF_LIB: the mutation tests point this at deliberately broken
+        # builds of the oracle to show that the pins notice.
+        lib = ctypes.CDLL(os.environ.get("PSOPS_REF_LIB") or build())
         lib.psops_ref_philox4x32_10.argtypes = [_u32p, _u32p, _u32p]
         lib.psops_ref_philox4x32_10.restype = None
         lib.psops_ref_uniform.argtypes = [ctypes.c_uint32]
