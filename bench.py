@@ -287,7 +287,7 @@ def run_psops(args):
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": f"{w.name}: K={w.K} particles x N={w.N} fp32 ({w.note}), "
                                f"omega={w.omega}, c1={w.c1}, c2={w.c2}, lambda={w.lam}, seed={w.seed}",
-                   "K": w.K, "N": w.N, "replicas": ranks.world,
+                   "K": w.K, "N": w.N, "ld": w.ld, "replicas": ranks.world,
                    "l2": "state (12*K*N bytes) exceeds L2; no flush needed",
                    "parallelism": "replicas only"},
         "clocks": sampler.report(),
@@ -323,6 +323,44 @@ def ncu_traffic(w):
     return NCU_TRAFFIC["bytes_per_particle_element"] * w.K * w.N
 
 
+def graph_us_per_sync(w, dev, replays=20):
+    """All S syncs of a small workload recorded into one CUDA graph (losses read
+    from the device table, step counter kept on the device) and replayed:
+    device time per sync without the host's launch cost."""
+    import torch
+    from paper_2009_03816_b200 import workloads
+    stream = torch.cuda.Stream(dev)
+    with torch.cuda.stream(stream):
+        sw = make_swarm(w, dev)
+        table = torch.from_numpy(workloads.losses(w)).to(dev)
+    stream.synchronize()
+    sw.close()
+    from paper_2009_03816_b200 import binding
+    sw = binding.Swarm(sw.x, sw.v, sw.pbest, N=w.N, m_max=w.omega, m_min=w.omega, c1=w.c1, c2=w.c2,
+                       seed=w.seed, stream=stream.cuda_stream)
+    rows = [table[s] for s in range(table.shape[0])]
+    with torch.cuda.stream(stream):
+        sw.set_losses(rows[0])
+        sw.sync(0, w.lam)
+    stream.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        for r in rows:
+            sw.set_losses(r)
+            sw.sync(0, w.lam)
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            graph.replay()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(replays):
+            graph.replay()
+        e1.record()
+    stream.synchronize()
+    sw.close()
+    return e0.elapsed_time(e1) * 1e3 / (replays * len(rows))
+
+
 def other_rows(args, dev, ranks, peak):
     """The remaining rows of the path, timed the same way (device-resident)."""
     import torch
@@ -353,7 +391,8 @@ def other_rows(args, dev, ranks, peak):
             ws = workloads.CONFIGS[name]
             sw, sec, _, _ = time_sync_workload(ws, dev, 200, 10, ranks)
             rows[name + "_sync"] = {"us_per_step": sec / 200 * 1e6, "value": ws.K * ws.N * 200 / sec,
-                                    "unit": UNIT, "note": "launch-bound / L2-resident"}
+                                    "unit": UNIT, "note": "small case: host launch rate / L2-resident",
+                                    "us_per_step_cuda_graph": graph_us_per_sync(ws, dev)}
             sw.close()
             del sw
     except Exception as exc:  # report, do not lose the headline line

@@ -99,7 +99,10 @@ int psops_create(psops_ctx **out, const psops_config *cfg,
  * Hand in the K current training losses (the fitness of Table I; lower is
  * better).  on_device == 0: host pointer, checked for NaN (ENAN) and copied
  * before the call returns to the stream (the buffer may be reused at once).
- * on_device != 0: device pointer, copied on the stream, not inspected.
+ * on_device != 0: device pointer (4-byte aligned), not inspected and not
+ * copied now: the selection kernel of the next psops_sync reads it on the
+ * stream (and keeps a copy), so the buffer must stay valid and unchanged until
+ * that sync has run.
  */
 int psops_set_losses(psops_ctx *ctx, const float *losses, int on_device);
 
@@ -118,7 +121,11 @@ int psops_set_losses(psops_ctx *ctx, const float *losses, int on_device);
  *      w' = w + v'.
  * If a quadratic fitness is attached (psops_set_quadratic) the losses of the
  * NEW weights are evaluated in the same pass and become the losses of the next
- * sync.  Enqueues work only; the sync counter advances by one.
+ * sync.  Enqueues work only; the sync counter advances by one.  The counter
+ * lives in device memory and is advanced by the selection kernel itself, so a
+ * psops_sync recorded into a CUDA graph (with the losses in a device buffer,
+ * see psops_set_losses) keeps walking the random stream when the graph is
+ * replayed; t_iter and lambda are then the ones given at capture.
  * Errors: EINVAL (t_iter < 0, lambda < 1 or not finite), ESTATE (no losses
  * yet), ECUDA.
  */

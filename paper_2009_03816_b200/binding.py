@@ -267,6 +267,7 @@ class Swarm:
             losses = np.ascontiguousarray(losses, dtype=np.float32)
         count = losses.size if isinstance(losses, np.ndarray) else losses.numel()
         assert count == self.K
+        self._loss_ref = losses        # a device buffer is read by the next sync: keep it alive
         psops_set_losses(self.ctx, losses)
 
     def sync(self, t_iter=0, lam=1.0):

@@ -20,6 +20,7 @@
 #include <cuda_runtime.h>
 
 #include <cmath>
+#include <cstddef>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -36,7 +37,10 @@ namespace {
 // Result of the selection kernel, read by the update kernel.
 struct SyncDesc {
     int      g;                 // index of the gBest particle (Algorithm 3)
-    int      pad[3];
+    uint32_t step;              // sync counter s of the sync in progress (Philox counter word 2)
+    uint32_t next_step;         // s of the next sync; advanced by the selection kernel so that a
+                                // captured-and-replayed sync still walks the random stream
+    int      pad;
     uint32_t improved[PSOPS_MAX_K / 32];   // bit i: loss_i < pBest_loss_i
 };
 
@@ -51,11 +55,35 @@ struct UpdateParams {
     long long tiles;            // ceil(N / 128)
     int K;
     float m, k1, k2;            // inertia, c1/lambda, c2/lambda
-    uint32_t step;              // sync counter s
     uint32_t rk[20];            // Philox round keys, rk[2r], rk[2r+1]
 };
 
-constexpr int kUpdateThreads = 256;
+// Launch shape of the streaming kernels; the defaults are the measured best on
+// B200 and can be overridden at build time for tuning sweeps.
+#ifndef PSOPS_UPDATE_THREADS
+#define PSOPS_UPDATE_THREADS 256
+#endif
+#ifndef PSOPS_UPDATE_UNROLL
+#define PSOPS_UPDATE_UNROLL 4          // particles in flight per thread; must divide 32
+#endif
+#ifndef PSOPS_UPDATE_QUADS
+#define PSOPS_UPDATE_QUADS 1           // quads per thread, one block-width apart
+#endif
+#ifndef PSOPS_FITNESS_UNROLL
+#define PSOPS_FITNESS_UNROLL 2         // particles in flight when the fitness is fused in
+#endif
+#ifndef PSOPS_FITNESS_QUADS
+#define PSOPS_FITNESS_QUADS 1
+#endif
+#ifndef PSOPS_UPDATE_MIN_BLOCKS
+#define PSOPS_UPDATE_MIN_BLOCKS 0      // >0: resident blocks per SM the register allocation must allow
+#endif
+#if PSOPS_UPDATE_MIN_BLOCKS > 0
+#define PSOPS_UPDATE_BOUNDS __launch_bounds__(PSOPS_UPDATE_THREADS, PSOPS_UPDATE_MIN_BLOCKS)
+#else
+#define PSOPS_UPDATE_BOUNDS __launch_bounds__(PSOPS_UPDATE_THREADS)
+#endif
+constexpr int kUpdateThreads = PSOPS_UPDATE_THREADS;
 constexpr int kFinalizeThreads = 1024;     // = number of level-2 slots
 constexpr int kTileElems = 128;            // one warp x one quad per lane
 
@@ -167,14 +195,19 @@ __device__ __forceinline__ bool beats(const Candidate &a, const Candidate &b)
 }
 
 __global__ void __launch_bounds__(PSOPS_MAX_K)
-psops_select_kernel(const float *__restrict__ loss, float *__restrict__ pbest_loss,
+psops_select_kernel(const float *loss, float *loss_keep, float *__restrict__ pbest_loss,
                     SyncDesc *__restrict__ desc, int K)
 {
+    // Let the update kernel that follows in the stream start its prologue; it
+    // waits for this grid to finish before it reads the descriptor.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
     __shared__ Candidate warp_best[PSOPS_MAX_K / 32];
     const int i = threadIdx.x;
     const int lane = i & 31, warp = i >> 5;
     const bool live = i < K;
     const float li = live ? loss[i] : 0.0f;
+    if (live) loss_keep[i] = li;             // the context's own copy (loss may be the caller's buffer)
 
     // pBest branch: strict "<" so that an equal loss never replaces pBest.
     const bool improved = live && (li < pbest_loss[i]);
@@ -201,91 +234,121 @@ psops_select_kernel(const float *__restrict__ loss, float *__restrict__ pbest_lo
         for (int w = 1; w < warps; ++w)
             if (beats(warp_best[w], c)) c = warp_best[w];
         desc->g = c.idx;
+        const uint32_t s_now = desc->next_step;
+        desc->step = s_now;
+        desc->next_step = s_now + 1u;
     }
 }
 
 // ---------------------------------------------------------------------------
 // Kernel (b): fused update (Eq. 6, Eq. 7 and the pBest copy of Algorithm 1),
 // optionally with the fitness of the new weights (levels 0 and 1).
-// Thread -> quad q (elements 4q..4q+3) for all K particles; a warp covers one
-// 128-element tile.  U particles are in flight per thread.
+// A thread owns Q quads (quad q = elements 4q..4q+3), one block-width apart,
+// for all K particles; a warp covers one 128-element tile per quad slot.
+// U particles x Q quads are in flight per thread: U*Q*3 independent 128-bit
+// loads before the first use.  Q > 1 makes every block stream a longer
+// contiguous piece of each row, which is what DRAM and the TLB like when K
+// rows x 3 arrays are all being walked at once.
 // ---------------------------------------------------------------------------
-template <bool ALIGNED, bool FITNESS, int U>
-__global__ void __launch_bounds__(kUpdateThreads)
+template <bool ALIGNED, bool FITNESS, int U, int Q>
+__global__ void PSOPS_UPDATE_BOUNDS
 psops_update_kernel(const __grid_constant__ UpdateParams P)
 {
-    const long long q = P.q_begin + (long long)blockIdx.x * kUpdateThreads + threadIdx.x;
-    const bool active = q < P.q_end;
-    if (!FITNESS && !active) return;         // with FITNESS whole warps stay for the shuffles
+    const long long q0 = P.q_begin + (long long)blockIdx.x * (kUpdateThreads * Q) + threadIdx.x;
+    // Launched with programmatic stream serialisation right behind the selection
+    // kernel: everything that kernel wrote is visible after this wait (a no-op
+    // for an ordinary launch).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (!FITNESS && q0 >= P.q_end) return;   // with FITNESS whole warps stay for the shuffles
 
-    const long long d0 = q * 4;
-    int nvalid = 0;
-    if (active && d0 < P.N) nvalid = (P.N - d0 >= 4) ? 4 : (int)(P.N - d0);
+    bool active[Q];
+    int nvalid[Q];
+    size_t col[Q];                           // element offset of quad slot j inside a row
+#pragma unroll
+    for (int j = 0; j < Q; ++j) {
+        const long long q = q0 + (long long)j * kUpdateThreads;
+        const long long d0 = q * 4;
+        active[j] = q < P.q_end;
+        nvalid[j] = 0;
+        if (active[j] && d0 < P.N) nvalid[j] = (P.N - d0 >= 4) ? 4 : (int)(P.N - d0);
+        col[j] = (size_t)d0;
+    }
 
     // gBest = row g as it is BEFORE this sync overwrites it; this thread is the
-    // only writer of these four elements, so reading them first is enough.
+    // only writer of these elements, so reading them first is enough.
     const int g = P.desc->g;
-    float gb[4];
-    load_quad_cached<ALIGNED>(P.x + (size_t)g * (size_t)P.ld + d0, nvalid, gb);
-    if (P.gbest_copy != nullptr) store_quad<ALIGNED>(P.gbest_copy + d0, nvalid, gb);
-
-    float dv[4] = {0.f, 0.f, 0.f, 0.f}, tv[4] = {0.f, 0.f, 0.f, 0.f};
-    if (FITNESS) {
-        load_quad_cached<ALIGNED>(P.dvec + d0, nvalid, dv);
-        load_quad_cached<ALIGNED>(P.tvec + d0, nvalid, tv);
+    const uint32_t step = P.desc->step;
+    float gb[Q][4];
+    float dv[Q][4], tv[Q][4];
+#pragma unroll
+    for (int j = 0; j < Q; ++j) {
+        load_quad_cached<ALIGNED>(P.x + (size_t)g * (size_t)P.ld + col[j], nvalid[j], gb[j]);
+        if (P.gbest_copy != nullptr) store_quad<ALIGNED>(P.gbest_copy + col[j], nvalid[j], gb[j]);
+        if (FITNESS) {
+            load_quad_cached<ALIGNED>(P.dvec + col[j], nvalid[j], dv[j]);
+            load_quad_cached<ALIGNED>(P.tvec + col[j], nvalid[j], tv[j]);
+        }
     }
 
     // Philox counter word 0 = element >> 1: 2q for elements 4q, 4q+1 and
     // 2q + 1 for elements 4q+2, 4q+3.
-    const uint32_t pair0 = (uint32_t)(2 * q);
+    const uint32_t pair0 = (uint32_t)(2 * q0);
 
-    size_t row = (size_t)d0;                 // offset of this quad in row i
+    size_t row = 0;                          // offset of row i0
     uint32_t impw = 0;
     for (int i0 = 0; i0 < P.K; i0 += U) {
         if ((i0 & 31) == 0) impw = P.desc->improved[i0 >> 5];
 
-        float xo[U][4], vo[U][4], pp[U][4];
+        float xo[U][Q][4], vo[U][Q][4], pp[U][Q][4];
         bool imp[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int i = i0 + u;
             imp[u] = (impw >> (i & 31)) & 1u;
             if (i < P.K) {
-                const size_t at = row + (size_t)u * (size_t)P.ld;
-                load_quad<ALIGNED>(P.x + at, nvalid, xo[u]);
-                load_quad<ALIGNED>(P.v + at, nvalid, vo[u]);
-                if (!imp[u]) load_quad<ALIGNED>(P.p + at, nvalid, pp[u]);
+#pragma unroll
+                for (int j = 0; j < Q; ++j) {
+                    const size_t at = row + (size_t)u * (size_t)P.ld + col[j];
+                    load_quad<ALIGNED>(P.x + at, nvalid[j], xo[u][j]);
+                    load_quad<ALIGNED>(P.v + at, nvalid[j], vo[u][j]);
+                    if (!imp[u]) load_quad<ALIGNED>(P.p + at, nvalid[j], pp[u][j]);
+                }
             }
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int i = i0 + u;
             if (i < P.K) {
-                const size_t at = row + (size_t)u * (size_t)P.ld;
-                uint32_t ra[4], rb[4];
-                philox4x32_10(pair0, (uint32_t)i, P.step, 0u, P.rk, ra);
-                philox4x32_10(pair0 + 1u, (uint32_t)i, P.step, 0u, P.rk, rb);
-                const uint32_t w1[4] = {ra[0], ra[2], rb[0], rb[2]};   // r1 of elements 0..3
-                const uint32_t w2[4] = {ra[1], ra[3], rb[1], rb[3]};   // r2 of elements 0..3
-                float vn[4], xn[4];
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const float pbest = imp[u] ? xo[u][e] : pp[u][e];  // pBest_i = w_i if improved
-                    const float dl = __fsub_rn(pbest, xo[u][e]);
-                    const float dg = __fsub_rn(gb[e], xo[u][e]);
-                    const float t1 = __fmul_rn(P.k1, uniform24(w1[e]));
-                    const float t2 = __fmul_rn(P.k2, uniform24(w2[e]));
-                    const float a0 = __fmul_rn(P.m, vo[u][e]);
-                    vn[e] = __fmaf_rn(t2, dg, __fmaf_rn(t1, dl, a0));  // Eq. 6
-                    xn[e] = __fadd_rn(xo[u][e], vn[e]);                 // Eq. 7
-                }
-                store_quad<ALIGNED>(P.v + at, nvalid, vn);
-                store_quad<ALIGNED>(P.x + at, nvalid, xn);
-                if (imp[u]) store_quad<ALIGNED>(P.p + at, nvalid, xo[u]);
-                if (FITNESS) {
-                    const double w = fitness_tile_sum(xn, dv, tv, nvalid);
-                    if ((threadIdx.x & 31) == 0 && active)   // q_end is a whole number of tiles
-                        P.partials[(size_t)i * (size_t)P.tiles + (size_t)(q >> 5)] = w;
+                for (int j = 0; j < Q; ++j) {
+                    const size_t at = row + (size_t)u * (size_t)P.ld + col[j];
+                    const uint32_t pair = pair0 + (uint32_t)(2 * j * kUpdateThreads);
+                    uint32_t ra[4], rb[4];
+                    philox4x32_10(pair, (uint32_t)i, step, 0u, P.rk, ra);
+                    philox4x32_10(pair + 1u, (uint32_t)i, step, 0u, P.rk, rb);
+                    const uint32_t w1[4] = {ra[0], ra[2], rb[0], rb[2]};   // r1 of elements 0..3
+                    const uint32_t w2[4] = {ra[1], ra[3], rb[1], rb[3]};   // r2 of elements 0..3
+                    float vn[4], xn[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float w = xo[u][j][e];
+                        const float pbest = imp[u] ? w : pp[u][j][e];      // pBest_i = w_i if improved
+                        const float dl = __fsub_rn(pbest, w);
+                        const float dg = __fsub_rn(gb[j][e], w);
+                        const float t1 = __fmul_rn(P.k1, uniform24(w1[e]));
+                        const float t2 = __fmul_rn(P.k2, uniform24(w2[e]));
+                        const float a0 = __fmul_rn(P.m, vo[u][j][e]);
+                        vn[e] = __fmaf_rn(t2, dg, __fmaf_rn(t1, dl, a0));  // Eq. 6
+                        xn[e] = __fadd_rn(w, vn[e]);                        // Eq. 7
+                    }
+                    store_quad<ALIGNED>(P.v + at, nvalid[j], vn);
+                    store_quad<ALIGNED>(P.x + at, nvalid[j], xn);
+                    if (imp[u]) store_quad<ALIGNED>(P.p + at, nvalid[j], xo[u][j]);
+                    if (FITNESS) {
+                        const double wsum = fitness_tile_sum(xn, dv[j], tv[j], nvalid[j]);
+                        if ((threadIdx.x & 31) == 0 && active[j])   // q_end is a whole number of tiles
+                            P.partials[(size_t)i * (size_t)P.tiles + (col[j] >> 7)] = wsum;
+                    }
                 }
             }
         }
@@ -433,6 +496,7 @@ struct psops_ctx {
     float *x, *v, *p;
     char *ws;
     float *d_losses, *d_pbest_loss, *d_gbest;
+    const float *loss_src;             // where the next selection reads the losses: d_losses or the caller's device buffer
     SyncDesc *d_desc;
     double *d_partials;
     const float *dvec, *tvec;
@@ -443,7 +507,7 @@ struct psops_ctx {
     bool aligned;
     bool have_losses;
     bool synced_once;
-    uint32_t step;
+    uint32_t step;                     // syncs enqueued through this context (the stream's own counter is on the device)
     long long quads, tiles;
     int64_t launches;
     char err[256];
@@ -485,15 +549,36 @@ void fill_round_keys(uint64_t seed, uint32_t (&rk)[20])
 int launch_select(psops_ctx *ctx)
 {
     const int threads = (int)round_up((size_t)ctx->cfg.K, 32);
-    psops_select_kernel<<<1, threads, 0, ctx->stream>>>(ctx->d_losses, ctx->d_pbest_loss,
+    psops_select_kernel<<<1, threads, 0, ctx->stream>>>(ctx->loss_src, ctx->d_losses, ctx->d_pbest_loss,
                                                         ctx->d_desc, ctx->cfg.K);
+    ctx->loss_src = ctx->d_losses;     // the kernel keeps a copy there
     return check_launch(ctx, "psops_select_kernel");
 }
 
-constexpr int kUnroll = 4;
+constexpr int kUnroll = PSOPS_UPDATE_UNROLL, kQuads = PSOPS_UPDATE_QUADS;
+constexpr int kFitUnroll = PSOPS_FITNESS_UNROLL, kFitQuads = PSOPS_FITNESS_QUADS;
+static_assert(32 % kUnroll == 0 && 32 % kFitUnroll == 0, "the improved mask is reloaded every 32 particles");
+static_assert(kUpdateThreads % 32 == 0, "a warp must cover whole 128-element tiles");
+
+template <typename Kernel>
+cudaError_t launch_update_kernel(Kernel kernel, unsigned blocks, cudaStream_t stream, bool after_select,
+                                 const UpdateParams &P)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(blocks, 1, 1);
+    cfg.blockDim = dim3(kUpdateThreads, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = after_select ? 1 : 0;   // overlap the launch with the selection kernel in front of it
+    return cudaLaunchKernelEx(&cfg, kernel, P);
+}
 
 int launch_update(psops_ctx *ctx, float m, float k1, float k2, long long q_begin,
-                  long long q_end, bool fitness, cudaStream_t stream)
+                  long long q_end, bool fitness, cudaStream_t stream, bool after_select = false)
 {
     if (q_end <= q_begin) return PSOPS_OK;
     UpdateParams P{};
@@ -506,17 +591,19 @@ int launch_update(psops_ctx *ctx, float m, float k1, float k2, long long q_begin
     P.tiles = ctx->tiles;
     P.K = ctx->cfg.K;
     P.m = m; P.k1 = k1; P.k2 = k2;
-    P.step = ctx->step;
     fill_round_keys(ctx->cfg.seed, P.rk);
     const long long span = q_end - q_begin;
-    const unsigned blocks = (unsigned)((span + kUpdateThreads - 1) / kUpdateThreads);
+    const int per_block = kUpdateThreads * (fitness ? kFitQuads : kQuads);
+    const unsigned blocks = (unsigned)((span + per_block - 1) / per_block);
+    cudaError_t e;
     if (ctx->aligned) {
-        if (fitness) psops_update_kernel<true, true, kUnroll><<<blocks, kUpdateThreads, 0, stream>>>(P);
-        else         psops_update_kernel<true, false, kUnroll><<<blocks, kUpdateThreads, 0, stream>>>(P);
+        if (fitness) e = launch_update_kernel(psops_update_kernel<true, true, kFitUnroll, kFitQuads>, blocks, stream, after_select, P);
+        else         e = launch_update_kernel(psops_update_kernel<true, false, kUnroll, kQuads>, blocks, stream, after_select, P);
     } else {
-        if (fitness) psops_update_kernel<false, true, kUnroll><<<blocks, kUpdateThreads, 0, stream>>>(P);
-        else         psops_update_kernel<false, false, kUnroll><<<blocks, kUpdateThreads, 0, stream>>>(P);
+        if (fitness) e = launch_update_kernel(psops_update_kernel<false, true, kFitUnroll, kFitQuads>, blocks, stream, after_select, P);
+        else         e = launch_update_kernel(psops_update_kernel<false, false, kUnroll, kQuads>, blocks, stream, after_select, P);
     }
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "psops_update_kernel launch");
     return check_launch(ctx, "psops_update_kernel");
 }
 
@@ -524,6 +611,7 @@ int launch_finalize(psops_ctx *ctx)
 {
     psops_fitness_finalize_kernel<<<ctx->cfg.K, kFinalizeThreads, 0, ctx->stream>>>(
         ctx->d_partials, ctx->d_losses, ctx->tiles);
+    ctx->loss_src = ctx->d_losses;
     return check_launch(ctx, "psops_fitness_finalize_kernel");
 }
 
@@ -608,6 +696,7 @@ int psops_create(psops_ctx **out, const psops_config *cfg, float *d_x, float *d_
     ctx->x = d_x; ctx->v = d_v; ctx->p = d_pbest;
     ctx->ws = (char *)d_workspace;
     ctx->d_losses = (float *)(ctx->ws + lay.off_losses);
+    ctx->loss_src = ctx->d_losses;
     ctx->d_pbest_loss = (float *)(ctx->ws + lay.off_pbest_loss);
     ctx->d_desc = (SyncDesc *)(ctx->ws + lay.off_desc);
     ctx->d_gbest = (cfg->flags & PSOPS_KEEP_GBEST) ? (float *)(ctx->ws + lay.off_gbest) : nullptr;
@@ -648,13 +737,15 @@ int psops_set_losses(psops_ctx *ctx, const float *losses, int on_device)
     if (ctx == nullptr || losses == nullptr) return PSOPS_EINVAL;
     const size_t bytes = sizeof(float) * (size_t)ctx->cfg.K;
     if (on_device) {
-        PSOPS_CUDA(ctx, cudaMemcpyAsync(ctx->d_losses, losses, bytes, cudaMemcpyDeviceToDevice, ctx->stream));
+        if (((uintptr_t)losses & 3u) != 0) return PSOPS_EALIGN;
+        ctx->loss_src = losses;        // read (and copied) by the selection kernel of the next sync
     } else {
         const int rc = check_host_losses(losses, ctx->cfg.K);
         if (rc != PSOPS_OK) return rc;
         // The source may be pageable and may be reused at once: wait for the copy.
         PSOPS_CUDA(ctx, cudaMemcpyAsync(ctx->d_losses, losses, bytes, cudaMemcpyHostToDevice, ctx->stream));
         PSOPS_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+        ctx->loss_src = ctx->d_losses;
     }
     ctx->have_losses = true;
     return PSOPS_OK;
@@ -675,7 +766,7 @@ int psops_sync(psops_ctx *ctx, int64_t t_iter, float lambda)
     // With the fused fitness every warp of a tile must be whole: round the
     // quad range up to a tile; quads past the end contribute +0.0.
     const long long q_end = fitness ? ctx->tiles * 32 : ctx->quads;
-    rc = launch_update(ctx, m, k1, k2, 0, q_end, fitness, ctx->stream);
+    rc = launch_update(ctx, m, k1, k2, 0, q_end, fitness, ctx->stream, /*after_select=*/true);
     if (rc != PSOPS_OK) return rc;
     if (fitness) {
         rc = launch_finalize(ctx);
@@ -711,6 +802,7 @@ int psops_sync_host(psops_ctx *ctx, const float *h_x_in, int64_t h_in_ld, const 
     // Losses and selection first: the update of any element range needs them.
     PSOPS_CUDA(ctx, cudaMemcpyAsync(ctx->d_losses, h_losses, sizeof(float) * (size_t)K,
                                     cudaMemcpyHostToDevice, ctx->stream));
+    ctx->loss_src = ctx->d_losses;
     ctx->have_losses = true;
     rc = launch_select(ctx);
     if (rc != PSOPS_OK) return rc;
@@ -839,7 +931,7 @@ int psops_get_losses(psops_ctx *ctx, float *dst, int dst_on_device)
 {
     if (ctx == nullptr || dst == nullptr) return PSOPS_EINVAL;
     if (!ctx->have_losses) return PSOPS_ESTATE;
-    PSOPS_CUDA(ctx, cudaMemcpyAsync(dst, ctx->d_losses, sizeof(float) * (size_t)ctx->cfg.K,
+    PSOPS_CUDA(ctx, cudaMemcpyAsync(dst, ctx->loss_src, sizeof(float) * (size_t)ctx->cfg.K,
                                     dst_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost,
                                     ctx->stream));
     if (!dst_on_device) PSOPS_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
@@ -888,12 +980,16 @@ int psops_eval_quadratic(psops_ctx *ctx)
 int psops_get_state(psops_ctx *ctx, uint32_t *sync_step, float *pbest_loss)
 {
     if (ctx == nullptr) return PSOPS_EINVAL;
-    if (pbest_loss != nullptr) {
+    // The counter lives on the device (a replayed graph advances it without
+    // the host taking part), so read it from there.
+    SyncDesc host{};
+    PSOPS_CUDA(ctx, cudaMemcpyAsync(&host, ctx->d_desc, sizeof(SyncDesc), cudaMemcpyDeviceToHost, ctx->stream));
+    if (pbest_loss != nullptr)
         PSOPS_CUDA(ctx, cudaMemcpyAsync(pbest_loss, ctx->d_pbest_loss, sizeof(float) * (size_t)ctx->cfg.K,
                                         cudaMemcpyDeviceToHost, ctx->stream));
-        PSOPS_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
-    }
-    if (sync_step != nullptr) *sync_step = ctx->step;
+    PSOPS_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    ctx->step = host.next_step;
+    if (sync_step != nullptr) *sync_step = host.next_step;
     return PSOPS_OK;
 }
 
@@ -904,6 +1000,8 @@ int psops_set_state(psops_ctx *ctx, uint32_t sync_step, const float *pbest_loss)
         if (pbest_loss[i] != pbest_loss[i]) return PSOPS_ENAN;
     PSOPS_CUDA(ctx, cudaMemcpyAsync(ctx->d_pbest_loss, pbest_loss, sizeof(float) * (size_t)ctx->cfg.K,
                                     cudaMemcpyHostToDevice, ctx->stream));
+    PSOPS_CUDA(ctx, cudaMemcpyAsync(reinterpret_cast<char *>(ctx->d_desc) + offsetof(SyncDesc, next_step),
+                                    &sync_step, sizeof(uint32_t), cudaMemcpyHostToDevice, ctx->stream));
     PSOPS_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     ctx->step = sync_step;
     return PSOPS_OK;

@@ -155,7 +155,7 @@ def test_cfg2_full():
 
 def test_cfg3_scaled_with_ties():
     w = workloads.CONFIGS["cfg3"].scaled(N=300_002)
-    assert w.ld == 300_004
+    assert w.N % 4 == 2 and w.ld == 300_032          # ragged last quad, padded pitch
     assert _run_workload(w, every=9) == 0
 
 
@@ -294,8 +294,8 @@ def test_cfg5_full_size_two_syncs():
                         seed=w.seed, flags=PSOPS_QUADRATIC)
     gpu.set_quadratic(dd, dt)
     gpu.eval_quadratic()
-    ref = oracle.RefSwarm(x, v, p, m_max=w.omega, m_min=w.omega, t_max=1, c1=w.c1, c2=w.c2,
-                          seed=w.seed, nthreads=NTHREADS)
+    ref = oracle.RefSwarm(x[:, :w.N], v[:, :w.N], p[:, :w.N], m_max=w.omega, m_min=w.omega, t_max=1,
+                          c1=w.c1, c2=w.c2, seed=w.seed, nthreads=NTHREADS)
     del x, v, p
     loss = oracle.quadratic_losses(ref.x, d, t, nthreads=NTHREADS)
     cols = torch.from_numpy(workloads.sample_columns(w.N, 200_000, 5)).to(dev)
@@ -415,6 +415,47 @@ def test_deterministic_and_resumable():
     assert sa.info()[0] == sc.info()[0] and np.array_equal(sa.info()[2], sc.info()[2])
     sa.close()
     sc.close()
+
+
+def test_sync_recorded_in_a_cuda_graph_replays_with_a_running_step_counter():
+    w = workloads.CONFIGS["cfg1"].scaled(N=40_001, S=8)
+    x, v, p = workloads.state(w)
+    table = workloads.losses(w)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        t = [torch.from_numpy(a).cuda() for a in (x, v, p)]
+        lbuf = torch.zeros(w.K, device="cuda")
+    stream.synchronize()
+    sw = binding.Swarm(*t, N=w.N, m_max=w.omega, m_min=w.omega, c1=w.c1, c2=w.c2, seed=w.seed,
+                       stream=stream.cuda_stream)
+    ref = oracle.RefSwarm(x[:, :w.N], v[:, :w.N], p[:, :w.N], m_max=w.omega, m_min=w.omega, t_max=1,
+                          c1=w.c1, c2=w.c2, seed=w.seed)
+    # one eager sync first (also warms the launch path), then record one sync
+    with torch.cuda.stream(stream):
+        lbuf.copy_(torch.from_numpy(table[0]))
+        sw.set_losses(lbuf)
+        sw.sync()
+    ref.sync(table[0])
+    stream.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        sw.set_losses(lbuf)
+        sw.sync()
+    # capture only records: the state must be unchanged
+    assert assert_close(t[0].cpu().numpy()[:, :w.N], ref.x, "after capture") == 0
+    for s in range(1, w.S):
+        with torch.cuda.stream(stream):
+            lbuf.copy_(torch.from_numpy(table[s]))
+            graph.replay()
+        ref.sync(table[s])
+        stream.synchronize()
+        g, improved, pl = sw.info()
+        assert g == ref.g and np.array_equal(improved, ref.improved)
+        assert np.array_equal(pl.view(np.uint32), ref.pbest_loss.view(np.uint32))
+    for got, want, name in ((t[0], ref.x, "x"), (t[1], ref.v, "v"), (t[2], ref.p, "pbest")):
+        assert assert_close(got.cpu().numpy()[:, :w.N], want, name) == 0
+    assert sw.state()[0] == w.S                     # the device-side counter saw every replay
+    sw.close()
 
 
 def test_runs_on_a_side_stream_and_counts_launches():

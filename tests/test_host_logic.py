@@ -125,10 +125,11 @@ def test_workload_shapes_follow_the_recipes():
     c = workloads.CONFIGS
     assert [(c[n].K, c[n].N) for n in ("cfg1", "cfg2", "cfg3", "cfg4", "cfg5")] == [
         (4, 61_706), (8, 1_250_000), (16, 11_173_962), (32, 25_557_032), (8, 50_000_000)]
-    assert c["cfg1"].ld == 61_708 and c["cfg3"].ld == 11_173_964 and c["cfg4"].ld == 25_557_032
+    assert c["cfg1"].ld == 62_464 and c["cfg3"].ld == 11_174_912 and c["cfg4"].ld == 25_558_016
+    assert all(c[n].ld % 1024 == 0 and 0 <= c[n].ld - c[n].N < 1024 for n in c)
     w = c["cfg2"].scaled(N=10_001)
     x, v, p = workloads.state(w)
-    assert x.shape == (8, 10_004) and x.dtype == np.float32
+    assert x.shape == (8, 10_240) and x.dtype == np.float32
     assert np.array_equal(p, x) and not x[:, 10_001:].any()
     assert abs(float(x[:, :10_001].std()) - 0.02) < 1e-3 and abs(float(v[:, :10_001].std()) - 1e-3) < 1e-4
     x2, _, _ = workloads.state(w)
