@@ -316,7 +316,7 @@ def run_psops(args):
 def ncu_traffic(w):
     if not NCU_TRAFFIC["source_sha256"]:
         return None
-    src = os.path.join(ROOT, "paper_2009_03816_b200", "csrc", "psops.cu")
+    src = os.path.join(ROOT, "paper_2009_03816_b200", "csrc", "psops_kernels.cuh")
     with open(src, "rb") as fh:
         if hashlib.sha256(fh.read()).hexdigest() != NCU_TRAFFIC["source_sha256"]:
             return None

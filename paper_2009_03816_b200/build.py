@@ -12,7 +12,7 @@ import sys
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 SOURCES = [os.path.join(_HERE, "csrc", "psops.cu")]
-HEADERS = [os.path.join(_ROOT, "include", "psops.h")]
+HEADERS = [os.path.join(_ROOT, "include", "psops.h"), os.path.join(_HERE, "csrc", "psops_kernels.cuh")]
 LIBRARY = os.path.join(_HERE, "libpsops.so")
 
 NVCC_FLAGS = [

@@ -1,4 +1,4 @@
-// psops.cu -- sm_100a kernels and C ABI of the PSO-PS synchronisation stage.
+// psops.cu -- C ABI and host side of the PSO-PS synchronisation stage (kernels: psops_kernels.cuh).
 //
 // The paper's synchronisation stage (Algorithm 1, sync branch; Algorithm 3;
 // Eq. 5-7) over K particles stored as K flat fp32 rows in HBM.  The stage is a
@@ -28,414 +28,9 @@
 #include <new>
 #include <vector>
 
+#include "psops_kernels.cuh"
+
 namespace {
-
-// ---------------------------------------------------------------------------
-// Device-side data
-// ---------------------------------------------------------------------------
-
-// Result of the selection kernel, read by the update kernel.
-struct SyncDesc {
-    int      g;                 // index of the gBest particle (Algorithm 3)
-    uint32_t step;              // sync counter s of the sync in progress (Philox counter word 2)
-    uint32_t next_step;         // s of the next sync; advanced by the selection kernel so that a
-                                // captured-and-replayed sync still walks the random stream
-    int      pad;
-    uint32_t improved[PSOPS_MAX_K / 32];   // bit i: loss_i < pBest_loss_i
-};
-
-struct UpdateParams {
-    float *x, *v, *p;           // K rows of stride ld
-    float *gbest_copy;          // NULL or N floats
-    const float *dvec, *tvec;   // quadratic fitness vectors (FITNESS only)
-    double *partials;           // K x tiles tile sums (FITNESS only)
-    const SyncDesc *desc;
-    long long ld, N;
-    long long q_begin, q_end;   // quad range of this launch (quad = 4 elements)
-    long long tiles;            // ceil(N / 128)
-    int K;
-    float m, k1, k2;            // inertia, c1/lambda, c2/lambda
-    uint32_t rk[20];            // Philox round keys, rk[2r], rk[2r+1]
-};
-
-// Launch shape of the streaming kernels; the defaults are the measured best on
-// B200 and can be overridden at build time for tuning sweeps.
-#ifndef PSOPS_UPDATE_THREADS
-#define PSOPS_UPDATE_THREADS 256
-#endif
-#ifndef PSOPS_UPDATE_UNROLL
-#define PSOPS_UPDATE_UNROLL 4          // particles in flight per thread; must divide 32
-#endif
-#ifndef PSOPS_UPDATE_QUADS
-#define PSOPS_UPDATE_QUADS 1           // quads per thread, one block-width apart
-#endif
-#ifndef PSOPS_FITNESS_UNROLL
-#define PSOPS_FITNESS_UNROLL 2         // particles in flight when the fitness is fused in
-#endif
-#ifndef PSOPS_FITNESS_QUADS
-#define PSOPS_FITNESS_QUADS 1
-#endif
-#ifndef PSOPS_UPDATE_MIN_BLOCKS
-#define PSOPS_UPDATE_MIN_BLOCKS 0      // >0: resident blocks per SM the register allocation must allow
-#endif
-#if PSOPS_UPDATE_MIN_BLOCKS > 0
-#define PSOPS_UPDATE_BOUNDS __launch_bounds__(PSOPS_UPDATE_THREADS, PSOPS_UPDATE_MIN_BLOCKS)
-#else
-#define PSOPS_UPDATE_BOUNDS __launch_bounds__(PSOPS_UPDATE_THREADS)
-#endif
-constexpr int kUpdateThreads = PSOPS_UPDATE_THREADS;
-constexpr int kFinalizeThreads = 1024;     // = number of level-2 slots
-constexpr int kTileElems = 128;            // one warp x one quad per lane
-
-// Philox4x32-10 (Salmon et al., SC'11).  Round keys are precomputed on the
-// host: they are the same for every thread of a launch.
-__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2,
-                                              uint32_t c3, const uint32_t (&rk)[20],
-                                              uint32_t (&out)[4])
-{
-#pragma unroll
-    for (int r = 0; r < 10; ++r) {
-        const unsigned long long pa = (unsigned long long)0xD2511F53u * c0;
-        const unsigned long long pb = (unsigned long long)0xCD9E8D57u * c2;
-        const uint32_t n0 = (uint32_t)(pb >> 32) ^ c1 ^ rk[2 * r];
-        const uint32_t n2 = (uint32_t)(pa >> 32) ^ c3 ^ rk[2 * r + 1];
-        c1 = (uint32_t)pb;
-        c3 = (uint32_t)pa;
-        c0 = n0;
-        c2 = n2;
-    }
-    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
-}
-
-// 32 random bits -> uniform on the 2^24 grid of [0,1); both steps are exact.
-__device__ __forceinline__ float uniform24(uint32_t w)
-{
-    return __fmul_rn(__uint2float_rn(w >> 8), 0x1p-24f);
-}
-
-// Load / store of one quad.  nvalid = 4 on the vector path means a full
-// 128-bit access; anything else goes element by element under a bound.
-template <bool ALIGNED>
-__device__ __forceinline__ void load_quad(const float *ptr, int nvalid, float (&a)[4])
-{
-    if (ALIGNED && nvalid == 4) {
-        const float4 t = __ldcs(reinterpret_cast<const float4 *>(ptr));
-        a[0] = t.x; a[1] = t.y; a[2] = t.z; a[3] = t.w;
-    } else {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) a[e] = (e < nvalid) ? __ldcs(ptr + e) : 0.0f;
-    }
-}
-
-// Plain (cacheable) variant for data that several reads share (gBest row,
-// dvec, tvec).
-template <bool ALIGNED>
-__device__ __forceinline__ void load_quad_cached(const float *ptr, int nvalid, float (&a)[4])
-{
-    if (ALIGNED && nvalid == 4) {
-        const float4 t = *reinterpret_cast<const float4 *>(ptr);
-        a[0] = t.x; a[1] = t.y; a[2] = t.z; a[3] = t.w;
-    } else {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) a[e] = (e < nvalid) ? ptr[e] : 0.0f;
-    }
-}
-
-template <bool ALIGNED>
-__device__ __forceinline__ void store_quad(float *ptr, int nvalid, const float (&a)[4])
-{
-    if (ALIGNED && nvalid == 4) {
-        __stcs(reinterpret_cast<float4 *>(ptr), make_float4(a[0], a[1], a[2], a[3]));
-    } else {
-#pragma unroll
-        for (int e = 0; e < 4; ++e)
-            if (e < nvalid) __stcs(ptr + e, a[e]);
-    }
-}
-
-// Level 0 and level 1 of the canonical fitness sum for one quad per lane:
-// fp32 terms dvec*(e*e), widened, added left to right, then the xor butterfly
-// over the warp.  Every lane returns the tile sum.
-__device__ __forceinline__ double fitness_tile_sum(const float (&xn)[4], const float (&dv)[4],
-                                                   const float (&tv)[4], int nvalid)
-{
-    double q = 0.0;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        double term = 0.0;
-        if (e < nvalid) {
-            const float err = __fsub_rn(xn[e], tv[e]);
-            term = (double)__fmul_rn(dv[e], __fmul_rn(err, err));
-        }
-        q = (e == 0) ? term : __dadd_rn(q, term);
-    }
-#pragma unroll
-    for (int off = 16; off >= 1; off >>= 1)
-        q = __dadd_rn(q, __shfl_xor_sync(0xffffffffu, q, off));
-    return q;
-}
-
-// ---------------------------------------------------------------------------
-// Kernel (a): selection.  One block, blockDim = K rounded up to a warp.
-// g = argmin loss (lowest index among equal minima, NaN never beats a number);
-// improved_i = loss_i < pBest_loss_i; pBest_loss_i <- loss_i where improved.
-// (Algorithm 3; Algorithm 1, pBest branch.)
-// ---------------------------------------------------------------------------
-struct Candidate { float loss; int idx; };
-
-__device__ __forceinline__ bool beats(const Candidate &a, const Candidate &b)
-{
-    const bool an = a.loss != a.loss, bn = b.loss != b.loss;
-    if (an != bn) return bn;                 // a number beats a NaN
-    if (!an) {
-        if (a.loss < b.loss) return true;
-        if (b.loss < a.loss) return false;
-    }
-    return a.idx < b.idx;                    // equal (or both NaN): lowest index
-}
-
-__global__ void __launch_bounds__(PSOPS_MAX_K)
-psops_select_kernel(const float *loss, float *loss_keep, float *__restrict__ pbest_loss,
-                    SyncDesc *__restrict__ desc, int K)
-{
-    // Let the update kernel that follows in the stream start its prologue; it
-    // waits for this grid to finish before it reads the descriptor.
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-
-    __shared__ Candidate warp_best[PSOPS_MAX_K / 32];
-    const int i = threadIdx.x;
-    const int lane = i & 31, warp = i >> 5;
-    const bool live = i < K;
-    const float li = live ? loss[i] : 0.0f;
-    if (live) loss_keep[i] = li;             // the context's own copy (loss may be the caller's buffer)
-
-    // pBest branch: strict "<" so that an equal loss never replaces pBest.
-    const bool improved = live && (li < pbest_loss[i]);
-    if (improved) pbest_loss[i] = li;
-    const uint32_t word = __ballot_sync(0xffffffffu, improved);
-    if (lane == 0) desc->improved[warp] = word;
-
-    // argmin
-    Candidate c;
-    c.loss = li;
-    c.idx = live ? i : 0x7fffffff;
-    if (!live) c.loss = __int_as_float(0x7fc00000);      // NaN with the largest index: never wins
-#pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) {
-        Candidate o;
-        o.loss = __shfl_xor_sync(0xffffffffu, c.loss, off);
-        o.idx = __shfl_xor_sync(0xffffffffu, c.idx, off);
-        if (beats(o, c)) c = o;
-    }
-    if (lane == 0) warp_best[warp] = c;
-    __syncthreads();
-    if (i == 0) {
-        const int warps = (blockDim.x + 31) >> 5;
-        for (int w = 1; w < warps; ++w)
-            if (beats(warp_best[w], c)) c = warp_best[w];
-        desc->g = c.idx;
-        const uint32_t s_now = desc->next_step;
-        desc->step = s_now;
-        desc->next_step = s_now + 1u;
-    }
-}
-
-// ---------------------------------------------------------------------------
-// Kernel (b): fused update (Eq. 6, Eq. 7 and the pBest copy of Algorithm 1),
-// optionally with the fitness of the new weights (levels 0 and 1).
-// A thread owns Q quads (quad q = elements 4q..4q+3), one block-width apart,
-// for all K particles; a warp covers one 128-element tile per quad slot.
-// U particles x Q quads are in flight per thread: U*Q*3 independent 128-bit
-// loads before the first use.  Q > 1 makes every block stream a longer
-// contiguous piece of each row, which is what DRAM and the TLB like when K
-// rows x 3 arrays are all being walked at once.
-// ---------------------------------------------------------------------------
-template <bool ALIGNED, bool FITNESS, int U, int Q>
-__global__ void PSOPS_UPDATE_BOUNDS
-psops_update_kernel(const __grid_constant__ UpdateParams P)
-{
-    const long long q0 = P.q_begin + (long long)blockIdx.x * (kUpdateThreads * Q) + threadIdx.x;
-    // Launched with programmatic stream serialisation right behind the selection
-    // kernel: everything that kernel wrote is visible after this wait (a no-op
-    // for an ordinary launch).
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (!FITNESS && q0 >= P.q_end) return;   // with FITNESS whole warps stay for the shuffles
-
-    bool active[Q];
-    int nvalid[Q];
-    size_t col[Q];                           // element offset of quad slot j inside a row
-#pragma unroll
-    for (int j = 0; j < Q; ++j) {
-        const long long q = q0 + (long long)j * kUpdateThreads;
-        const long long d0 = q * 4;
-        active[j] = q < P.q_end;
-        nvalid[j] = 0;
-        if (active[j] && d0 < P.N) nvalid[j] = (P.N - d0 >= 4) ? 4 : (int)(P.N - d0);
-        col[j] = (size_t)d0;
-    }
-
-    // gBest = row g as it is BEFORE this sync overwrites it; this thread is the
-    // only writer of these elements, so reading them first is enough.
-    const int g = P.desc->g;
-    const uint32_t step = P.desc->step;
-    float gb[Q][4];
-    float dv[Q][4], tv[Q][4];
-#pragma unroll
-    for (int j = 0; j < Q; ++j) {
-        load_quad_cached<ALIGNED>(P.x + (size_t)g * (size_t)P.ld + col[j], nvalid[j], gb[j]);
-        if (P.gbest_copy != nullptr) store_quad<ALIGNED>(P.gbest_copy + col[j], nvalid[j], gb[j]);
-        if (FITNESS) {
-            load_quad_cached<ALIGNED>(P.dvec + col[j], nvalid[j], dv[j]);
-            load_quad_cached<ALIGNED>(P.tvec + col[j], nvalid[j], tv[j]);
-        }
-    }
-
-    // Philox counter word 0 = element >> 1: 2q for elements 4q, 4q+1 and
-    // 2q + 1 for elements 4q+2, 4q+3.
-    const uint32_t pair0 = (uint32_t)(2 * q0);
-
-    size_t row = 0;                          // offset of row i0
-    uint32_t impw = 0;
-    for (int i0 = 0; i0 < P.K; i0 += U) {
-        if ((i0 & 31) == 0) impw = P.desc->improved[i0 >> 5];
-
-        float xo[U][Q][4], vo[U][Q][4], pp[U][Q][4];
-        bool imp[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int i = i0 + u;
-            imp[u] = (impw >> (i & 31)) & 1u;
-            if (i < P.K) {
-#pragma unroll
-                for (int j = 0; j < Q; ++j) {
-                    const size_t at = row + (size_t)u * (size_t)P.ld + col[j];
-                    load_quad<ALIGNED>(P.x + at, nvalid[j], xo[u][j]);
-                    load_quad<ALIGNED>(P.v + at, nvalid[j], vo[u][j]);
-                    if (!imp[u]) load_quad<ALIGNED>(P.p + at, nvalid[j], pp[u][j]);
-                }
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int i = i0 + u;
-            if (i < P.K) {
-#pragma unroll
-                for (int j = 0; j < Q; ++j) {
-                    const size_t at = row + (size_t)u * (size_t)P.ld + col[j];
-                    const uint32_t pair = pair0 + (uint32_t)(2 * j * kUpdateThreads);
-                    uint32_t ra[4], rb[4];
-                    philox4x32_10(pair, (uint32_t)i, step, 0u, P.rk, ra);
-                    philox4x32_10(pair + 1u, (uint32_t)i, step, 0u, P.rk, rb);
-                    const uint32_t w1[4] = {ra[0], ra[2], rb[0], rb[2]};   // r1 of elements 0..3
-                    const uint32_t w2[4] = {ra[1], ra[3], rb[1], rb[3]};   // r2 of elements 0..3
-                    float vn[4], xn[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float w = xo[u][j][e];
-                        const float pbest = imp[u] ? w : pp[u][j][e];      // pBest_i = w_i if improved
-                        const float dl = __fsub_rn(pbest, w);
-                        const float dg = __fsub_rn(gb[j][e], w);
-                        const float t1 = __fmul_rn(P.k1, uniform24(w1[e]));
-                        const float t2 = __fmul_rn(P.k2, uniform24(w2[e]));
-                        const float a0 = __fmul_rn(P.m, vo[u][j][e]);
-                        vn[e] = __fmaf_rn(t2, dg, __fmaf_rn(t1, dl, a0));  // Eq. 6
-                        xn[e] = __fadd_rn(w, vn[e]);                        // Eq. 7
-                    }
-                    store_quad<ALIGNED>(P.v + at, nvalid[j], vn);
-                    store_quad<ALIGNED>(P.x + at, nvalid[j], xn);
-                    if (imp[u]) store_quad<ALIGNED>(P.p + at, nvalid[j], xo[u][j]);
-                    if (FITNESS) {
-                        const double wsum = fitness_tile_sum(xn, dv[j], tv[j], nvalid[j]);
-                        if ((threadIdx.x & 31) == 0 && active[j])   // q_end is a whole number of tiles
-                            P.partials[(size_t)i * (size_t)P.tiles + (col[j] >> 7)] = wsum;
-                    }
-                }
-            }
-        }
-        row += (size_t)U * (size_t)P.ld;
-    }
-}
-
-// ---------------------------------------------------------------------------
-// Kernel (c): parameter averaging (Section II-B, step 5).
-// ---------------------------------------------------------------------------
-template <bool ALIGNED, int U>
-__global__ void __launch_bounds__(kUpdateThreads)
-psops_average_kernel(float *__restrict__ x, long long ld, long long N, long long quads, int K)
-{
-    const long long q = (long long)blockIdx.x * kUpdateThreads + threadIdx.x;
-    if (q >= quads) return;
-    const long long d0 = q * 4;
-    const int nvalid = (N - d0 >= 4) ? 4 : (int)(N - d0);
-    const float kf = (float)K;
-
-    float acc[4];
-    load_quad<ALIGNED>(x + d0, nvalid, acc);
-    int k = 1;
-    for (; k < K; k += U) {
-        float t[U][4];
-#pragma unroll
-        for (int u = 0; u < U; ++u)
-            if (k + u < K) load_quad<ALIGNED>(x + (size_t)(k + u) * (size_t)ld + d0, nvalid, t[u]);
-#pragma unroll
-        for (int u = 0; u < U; ++u)
-            if (k + u < K) {
-#pragma unroll
-                for (int e = 0; e < 4; ++e) acc[e] = __fadd_rn(acc[e], t[u][e]);
-            }
-    }
-#pragma unroll
-    for (int e = 0; e < 4; ++e) acc[e] = __fdiv_rn(acc[e], kf);
-    for (k = 0; k < K; ++k) store_quad<ALIGNED>(x + (size_t)k * (size_t)ld + d0, nvalid, acc);
-}
-
-// ---------------------------------------------------------------------------
-// Kernel (d): stand-alone fitness tile sums (levels 0 and 1), and the level-2
-// finalisation shared with the fused path.
-// ---------------------------------------------------------------------------
-template <bool ALIGNED>
-__global__ void __launch_bounds__(kUpdateThreads)
-psops_fitness_tiles_kernel(const float *__restrict__ x, const float *__restrict__ dvec,
-                           const float *__restrict__ tvec, double *__restrict__ partials,
-                           long long ld, long long N, long long quads, long long tiles, int K)
-{
-    const long long q = (long long)blockIdx.x * kUpdateThreads + threadIdx.x;
-    const long long d0 = q * 4;
-    int nvalid = 0;
-    if (q < quads) nvalid = (N - d0 >= 4) ? 4 : (int)(N - d0);
-    if ((q >> 5) >= tiles) return;           // whole warp out of range
-    float dv[4], tv[4];
-    load_quad_cached<ALIGNED>(dvec + d0, nvalid, dv);
-    load_quad_cached<ALIGNED>(tvec + d0, nvalid, tv);
-    for (int i = 0; i < K; ++i) {
-        float xi[4];
-        load_quad<ALIGNED>(x + (size_t)i * (size_t)ld + d0, nvalid, xi);
-        const double w = fitness_tile_sum(xi, dv, tv, nvalid);
-        if ((threadIdx.x & 31) == 0) partials[(size_t)i * (size_t)tiles + (size_t)(q >> 5)] = w;
-    }
-}
-
-// One block per particle, thread tau = slot tau.
-__global__ void __launch_bounds__(kFinalizeThreads)
-psops_fitness_finalize_kernel(const double *__restrict__ partials, float *__restrict__ loss,
-                              long long tiles)
-{
-    __shared__ double group[kFinalizeThreads / 32];
-    const int i = blockIdx.x;
-    const double *row = partials + (size_t)i * (size_t)tiles;
-    double acc = 0.0;
-    for (long long m = threadIdx.x; m < tiles; m += kFinalizeThreads) acc = __dadd_rn(acc, row[m]);
-#pragma unroll
-    for (int off = 16; off >= 1; off >>= 1)
-        acc = __dadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, off));
-    if ((threadIdx.x & 31) == 0) group[threadIdx.x >> 5] = acc;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        double total = group[0];
-        for (int gq = 1; gq < kFinalizeThreads / 32; ++gq) total = __dadd_rn(total, group[gq]);
-        loss[i] = (float)total;
-    }
-}
 
 // ---------------------------------------------------------------------------
 // Host side
