@@ -15,6 +15,7 @@ from .psops_oracle import (  # noqa: F401
     philox4x32_10,
     quadratic_fitness,
     quadratic_losses,
+    ssgd,
     sync,
     uniform,
     update_element,

@@ -73,11 +73,15 @@ def _load():
             ctypes.c_float, ctypes.c_float, ctypes.c_float,
             ctypes.c_uint64, ctypes.c_uint32,
             _i64p, _f32p, ctypes.POINTER(ctypes.c_int), _u8p, _f32p,
+            _f32p, _f32p, ctypes.POINTER(ctypes.c_int),
             ctypes.c_int]
         lib.psops_ref_sync.restype = ctypes.c_int
         lib.psops_ref_average.argtypes = [ctypes.c_int, ctypes.c_int64,
                                           ctypes.c_int64, _f32p, ctypes.c_int]
         lib.psops_ref_average.restype = None
+        lib.psops_ref_ssgd.argtypes = [ctypes.c_int, ctypes.c_int64, ctypes.c_int64, _f32p,
+                                       _f32p, ctypes.c_int64, ctypes.c_float, ctypes.c_int]
+        lib.psops_ref_ssgd.restype = None
         lib.psops_ref_quadratic_fitness.argtypes = [_f32p, _f32p, _f32p,
                                                     ctypes.c_int64]
         lib.psops_ref_quadratic_fitness.restype = ctypes.c_float
@@ -149,9 +153,11 @@ def update_element(m, k1, k2, r1, r2, xo, vo, pp, gb):
 
 
 def sync(x, v, p, loss, pbest_loss, *, m_max, m_min, t, t_max, c1, c2, lam,
-         seed, s, elem_index=None, fixed_r=None, nthreads=1, want_gbest=False):
+         seed, s, elem_index=None, fixed_r=None, nthreads=1, want_gbest=False, history=None):
     """One synchronisation in place on x, v, p (2-D fp32, rows contiguous) and
-    pbest_loss (1-D fp32).  Returns (g, improved[K] bool, gbest row or None)."""
+    pbest_loss (1-D fp32).  Returns (g, improved[K] bool, gbest row or None).
+    history: None, or a dict {"row": n fp32, "loss": 1 fp32, "valid": 1 int32}
+    updated in place (gBest from the history of all particles)."""
     K, n, ld = _rows(x)
     assert _rows(v) == (K, n, ld) and _rows(p) == (K, n, ld)
     loss = np.ascontiguousarray(loss, dtype=np.float32)
@@ -175,7 +181,11 @@ def sync(x, v, p, loss, pbest_loss, *, m_max, m_min, t, t_max, c1, c2, lam,
         float(np.float32(m_max)), float(np.float32(m_min)), int(t), int(t_max),
         float(np.float32(c1)), float(np.float32(c2)), float(np.float32(lam)),
         int(seed), int(s), ei, fr, ctypes.byref(g), imp.ctypes.data_as(_u8p),
-        _f32(gb) if gb is not None else None, int(nthreads))
+        _f32(gb) if gb is not None else None,
+        _f32(history["row"]) if history else None,
+        _f32(history["loss"]) if history else None,
+        history["valid"].ctypes.data_as(ctypes.POINTER(ctypes.c_int)) if history else None,
+        int(nthreads))
     if rc != 0:
         raise MemoryError("psops_ref_sync: allocation failed")
     return int(g.value), imp.astype(bool), gb
@@ -184,6 +194,15 @@ def sync(x, v, p, loss, pbest_loss, *, m_max, m_min, t, t_max, c1, c2, lam,
 def average(x, nthreads=1) -> None:
     K, n, ld = _rows(x)
     _load().psops_ref_average(K, n, ld, x.ctypes.data_as(_f32p), int(nthreads))
+
+
+def ssgd(w, grad, alpha, nthreads=1) -> None:
+    """w (K rows) <- w[0] + (alpha / K) * sum_k grad[k], written to every row."""
+    K, n, ld = _rows(w)
+    Kg, ng, gld = _rows(grad)
+    assert (Kg, ng) == (K, n)
+    _load().psops_ref_ssgd(K, n, ld, w.ctypes.data_as(_f32p), grad.ctypes.data_as(_f32p), gld,
+                           float(np.float32(alpha)), int(nthreads))
 
 
 def quadratic_fitness(x, dvec, tvec) -> np.float32:
@@ -216,7 +235,7 @@ class RefSwarm:
     """
 
     def __init__(self, x, v, p, *, m_max, m_min, t_max, c1, c2, seed,
-                 elem_index=None, nthreads=1):
+                 elem_index=None, nthreads=1, history=False):
         self.x = np.array(x, dtype=np.float32, copy=True, order="C")
         self.v = np.array(v, dtype=np.float32, copy=True, order="C")
         self.p = np.array(p, dtype=np.float32, copy=True, order="C")
@@ -230,12 +249,17 @@ class RefSwarm:
         self.g = -1
         self.improved = np.zeros(self.K, dtype=bool)
         self.gbest = None
+        self.history = None
+        if history:
+            self.history = {"row": np.zeros(self.x.shape[1], np.float32),
+                            "loss": np.full(1, np.inf, np.float32),
+                            "valid": np.zeros(1, np.int32)}
 
     def sync(self, loss, t=0, lam=1.0, want_gbest=False):
         self.g, self.improved, self.gbest = sync(
             self.x, self.v, self.p, loss, self.pbest_loss, t=t, lam=lam,
             s=self.s, elem_index=self.elem_index, nthreads=self.nthreads,
-            want_gbest=want_gbest, **self.cfg)
+            want_gbest=want_gbest, history=self.history, **self.cfg)
         self.s += 1
         return self.g, self.improved
 

@@ -15,6 +15,8 @@
  *   - Eq. 6 / Eq. 7 velocity and position update        -> psops_ref_update_element
  *   - Algorithm 1, the synchronisation branch as a whole -> psops_ref_sync
  *   - Section II-B, parameter averaging, step 5          -> psops_ref_average
+ *   - Section II-B, synchronous SGD update               -> psops_ref_ssgd
+ *   - Section II-C, step 3 (gBest from history), as an option of psops_ref_sync
  * The random numbers r1, r2 of Eq. 6 come from Philox4x32-10 (Salmon, Moraes,
  * Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3", SC'11), written
  * here from the published round definition.
@@ -170,7 +172,15 @@ void psops_ref_update_element(float m, float k1, float k2, float r1, float r2,
  *                of one another once the losses are given)
  *   fixed_r      NULL, or {r1, r2} used for every draw (worked examples)
  *   g_out, improved_out   selection results (may be NULL)
- *   gbest_out    NULL or n floats: the gBest row, i.e. row g before the update
+ *   gbest_out    NULL or n floats: the gBest row that Eq. 6 used
+ *   hist_row, hist_loss, hist_valid
+ *                all NULL: gBest is the best particle of THIS iteration
+ *                (Algorithm 3).  All non-NULL: the standard-PSO variant
+ *                (Section II-C, step 3: gBest "from the history of all
+ *                particles"): the remembered row (n floats), its loss and a
+ *                0/1 flag, updated in place -- the current best replaces the
+ *                remembered one only on a strictly smaller loss (or when
+ *                nothing is remembered yet), and Eq. 6 uses the remembered row
  *   nthreads     >1 splits the element loop across OpenMP threads; the result
  *                is the same because every draw is a pure function of
  *                (seed, s, i, d)
@@ -183,6 +193,7 @@ int psops_ref_sync(int K, int64_t n, int64_t ld, float *x, float *v, float *p,
                    uint64_t seed, uint32_t s,
                    const int64_t *elem_index, const float *fixed_r,
                    int *g_out, uint8_t *improved_out, float *gbest_out,
+                   float *hist_row, float *hist_loss, int *hist_valid,
                    int nthreads)
 {
     /* schedule scalars */
@@ -200,6 +211,15 @@ int psops_ref_sync(int K, int64_t n, int64_t ld, float *x, float *v, float *p,
     /* gBest is the best particle's weights at this iteration: copy the row   */
     /* before anything is overwritten.                                        */
     memcpy(gb, x + (size_t)g * (size_t)ld, sizeof(float) * (size_t)n);
+    if (hist_row && hist_loss && hist_valid) {
+        if (!*hist_valid || loss[g] < *hist_loss) {
+            memcpy(hist_row, gb, sizeof(float) * (size_t)n);     /* new best in history */
+            *hist_loss = loss[g];
+            *hist_valid = 1;
+        } else {
+            memcpy(gb, hist_row, sizeof(float) * (size_t)n);     /* keep the remembered one */
+        }
+    }
 
     if (nthreads < 1) nthreads = 1;
 #pragma omp parallel for num_threads(nthreads) schedule(static)
@@ -243,6 +263,28 @@ void psops_ref_average(int K, int64_t n, int64_t ld, float *x, int nthreads)
         const float mean = acc / (float)K;
         for (int k = 0; k < K; ++k)
             x[(size_t)k * (size_t)ld + (size_t)j] = mean;
+    }
+}
+
+/* Synchronous SGD as the paper states it next to parameter averaging        */
+/* (Section II-B): w_{i+1} = w_i + (1/n) alpha sum_k grad_k, handed to every  */
+/* worker.  fp32: gradients summed in worker order, scale = alpha / n (one    */
+/* division), one product, one addition.  w holds the n workers' (identical   */
+/* or not) weights; the new weight is computed from worker 0's row.           */
+void psops_ref_ssgd(int K, int64_t n, int64_t ld, float *w, const float *grad,
+                    int64_t grad_ld, float alpha, int nthreads)
+{
+    if (nthreads < 1) nthreads = 1;
+    const float scale = alpha / (float)K;
+#pragma omp parallel for num_threads(nthreads) schedule(static)
+    for (int64_t j = 0; j < n; ++j) {
+        float acc = grad[j];
+        for (int k = 1; k < K; ++k)
+            acc = acc + grad[(size_t)k * (size_t)grad_ld + (size_t)j];
+        const float step = scale * acc;
+        const float wn = w[j] + step;
+        for (int k = 0; k < K; ++k)
+            w[(size_t)k * (size_t)ld + (size_t)j] = wn;
     }
 }
 

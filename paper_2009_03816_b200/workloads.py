@@ -38,6 +38,11 @@ class Workload:
     quadratic: bool = False  # fitness evaluated on device, no loss table
     lam: float = 1.0
     note: str = ""
+    # Table II style schedules (all zero / None: constant inertia omega, constant lambda)
+    m_min: float | None = None   # Eq. 5 lower inertia; m_max is `omega`
+    sync_period: int = 0         # `step` of Algorithm 1: training iterations between syncs
+    iters_per_epoch: int = 0     # training-set size / batch size
+    epochs: int = 0              # lambda = epoch index 1..epochs; t_max = epochs * iters_per_epoch
 
     @property
     def ld(self) -> int:
@@ -46,6 +51,26 @@ class Workload:
         128-bit kernels need; the 4-KiB pitch is worth a further ~4 % of HBM
         bandwidth on B200 (measured) for at most 4 KiB of padding per row."""
         return (self.N + 1023) // 1024 * 1024
+
+    @property
+    def m_max(self) -> float:
+        return self.omega
+
+    @property
+    def m_lo(self) -> float:
+        return self.omega if self.m_min is None else self.m_min
+
+    @property
+    def t_max(self) -> int:
+        return self.epochs * self.iters_per_epoch if self.epochs else 1
+
+    def schedule(self, s: int) -> tuple[int, float]:
+        """(t_iter, lambda) of sync s: Algorithm 1 syncs whenever t % step == 0,
+        t counting training iterations from 1; lambda is the 1-based epoch."""
+        if not self.sync_period:
+            return 0, self.lam
+        t = (s + 1) * self.sync_period
+        return t, float(min(self.epochs, 1 + (t - 1) // self.iters_per_epoch))
 
     def scaled(self, N: int, S: int | None = None) -> "Workload":
         """Same recipe at another vector length (parity cases that a CPU
@@ -70,6 +95,13 @@ CONFIGS = {
     "cfg5": Workload("cfg5", K=8, N=50_000_000, S=200, omega=0.7, c1=1.5, c2=1.5,
                      seed=5, sigma_x=1.0, sigma_v=0.0, quadratic=True,
                      note="quadratic fitness evaluated on device"),
+    # The paper's own settings (Table II: m 0.9 -> 0.3, c1 0.2, c2 0.9, lambda = epoch) on its
+    # LeNet/MNIST schedule: 60,000 samples / batch 256 = 234 iterations per epoch, 25 epochs,
+    # a sync every 10 iterations -> 585 syncs.  Only shapes and the schedule are used.
+    "cfg6": Workload("cfg6", K=8, N=61_706, S=585, omega=0.9, m_min=0.3, c1=0.2, c2=0.9,
+                     seed=6, sigma_x=0.05, sigma_v=0.0, loss_lo=0.1, loss_hi=2.5,
+                     sync_period=10, iters_per_epoch=234, epochs=25,
+                     note="Table II schedule on a LeNet-5-sized vector"),
 }
 
 

@@ -51,7 +51,21 @@ MUTANTS = [
     ("schedule sign", "(double)m_max\n             - (double)t", "(double)m_max\n             + (double)t"),
     ("schedule not clamped", "if (t > t_max) t = t_max;", ""),
     ("average divides by K-1", "acc / (float)K", "acc / (float)(K > 1 ? K - 1 : 1)"),
-    ("average counts row 0 twice", "for (int k = 1; k < K; ++k)\n            acc = acc", "for (int k = 0; k < K; ++k)\n            acc = acc"),
+    ("average counts row 0 twice", "for (int k = 1; k < K; ++k)\n            acc = acc + x[",
+     "for (int k = 0; k < K; ++k)\n            acc = acc + x["),
+    ("ssgd counts worker 0 twice", "for (int k = 1; k < K; ++k)\n            acc = acc + grad[",
+     "for (int k = 0; k < K; ++k)\n            acc = acc + grad["),
+    ("history: equal loss replaces the remembered best", "if (!*hist_valid || loss[g] < *hist_loss) {",
+     "if (!*hist_valid || loss[g] <= *hist_loss) {"),
+    ("history: empty memory not filled", "if (!*hist_valid || loss[g] < *hist_loss) {",
+     "if (loss[g] < *hist_loss) {"),
+    ("history: remembered row not used", "memcpy(gb, hist_row, sizeof(float) * (size_t)n);     /* keep", "/* keep"),
+    ("history: remembers the post-update row", "memcpy(hist_row, gb, sizeof(float) * (size_t)n);     /* new best in history */",
+     "/* new best in history */"),
+    ("ssgd not divided by the worker count", "const float scale = alpha / (float)K;", "const float scale = alpha;"),
+    ("ssgd subtracts", "const float wn = w[j] + step;", "const float wn = w[j] - step;"),
+    ("ssgd ignores the gradient stride", "acc = acc + grad[(size_t)k * (size_t)grad_ld + (size_t)j];",
+     "acc = acc + grad[(size_t)k * (size_t)ld + (size_t)j];"),
     ("fitness error not squared", "float e2 = e * e;", "float e2 = e;"),
     ("fitness uses tvec as weight", "float term = dvec[j] * e2;", "float term = tvec[j] * e2;"),
     ("fitness drops the last element of a quad", "a = a + quad_term(x, dvec, tvec, j + 3, N);", ""),

@@ -515,3 +515,126 @@ def test_pso_on_quadratic_converges_towards_minimiser():
     assert best_hist[-1] < 1e-6 * first
     best = sw.p[int(np.argmin(sw.pbest_loss))]
     assert np.abs(best - t).max() < 1e-2
+
+
+# --------------------------------------------------------------------------
+# gBest from the history of all particles (standard PSO, Section II-C step 3).
+# --------------------------------------------------------------------------
+def test_history_gbest_hand_worked_three_syncs():
+    """K=2, N=2, m=0.5, c1=0, c2=1, r2=0.5 -> v' = 0.5 v + 0.5 (gBest - w).
+    Sync 1: losses [1, 0.5] -> g=1, nothing remembered yet -> gBest=[0,4], loss 0.5.
+       p0: v'=0.5([0,4]-[2,0])=[-1,2], w'=[1,2];  p1: v'=0, w'=[0,4].
+    Sync 2: losses [0.75, 2] -> current best p0=[1,2] with 0.75 >= 0.5: gBest stays [0,4].
+       p0: v'=0.5[-1,2]+0.5([0,4]-[1,2])=[-1,2], w'=[0,4];  p1: v'=0, w'=[0,4].
+       (current-iteration gBest would give w'=[0.5,3] for both.)
+    Sync 3: losses [0.25, 1] -> 0.25 < 0.5: gBest <- p0's weights before the update = [0,4]."""
+    x = np.array([[2, 0], [0, 4]], np.float32)
+    for history, expect2 in ((True, [[0, 4], [0, 4]]), (False, [[0.5, 3], [0.5, 3]])):
+        sw = oracle.RefSwarm(x, np.zeros_like(x), x, m_max=0.5, m_min=0.5, t_max=1, c1=0.0, c2=1.0,
+                             seed=0, history=history)
+        kw = dict(m_max=0.5, m_min=0.5, t=0, t_max=1, c1=0.0, c2=1.0, lam=1.0, seed=0,
+                  fixed_r=np.array([0.5, 0.5], np.float32), history=sw.history, want_gbest=True)
+        g, _, gb = oracle.sync(sw.x, sw.v, sw.p, [1.0, 0.5], sw.pbest_loss, s=0, **kw)
+        assert g == 1 and gb.tolist() == [0, 4]
+        assert sw.x.tolist() == [[1, 2], [0, 4]] and sw.v.tolist() == [[-1, 2], [0, 0]]
+        g, _, gb = oracle.sync(sw.x, sw.v, sw.p, [0.75, 2.0], sw.pbest_loss, s=1, **kw)
+        assert g == 0
+        assert gb.tolist() == ([0, 4] if history else [1, 2])
+        assert sw.x.tolist() == expect2
+        if history:
+            assert sw.history["loss"][0] == np.float32(0.5) and sw.history["row"].tolist() == [0, 4]
+            g, _, gb = oracle.sync(sw.x, sw.v, sw.p, [0.25, 1.0], sw.pbest_loss, s=2, **kw)
+            assert g == 0 and sw.history["loss"][0] == np.float32(0.25)
+            assert gb.tolist() == [0, 4] and sw.history["row"].tolist() == [0, 4]
+
+
+def test_history_gbest_properties():
+    K, n = 5, 301
+    x, v, p = _random_swarm(K, n, 23)
+    rng = np.random.default_rng(5)
+    cur = oracle.RefSwarm(x, v, p, m_max=0.7, m_min=0.7, t_max=1, c1=1.5, c2=1.5, seed=3)
+    his = oracle.RefSwarm(x, v, p, m_max=0.7, m_min=0.7, t_max=1, c1=1.5, c2=1.5, seed=3, history=True)
+    # strictly decreasing minimum: the remembered best is always the current one
+    for s in range(5):
+        loss = (rng.random(K) + 10.0 - s).astype(np.float32)
+        cur.sync(loss)
+        his.sync(loss)
+        assert np.array_equal(cur.x, his.x) and np.array_equal(cur.v, his.v)
+        assert his.history["loss"][0] == loss.min()
+    # from now on nothing beats the remembered loss: the row must not move
+    kept = his.history["row"].copy()
+    kept_loss = his.history["loss"][0]
+    for s in range(4):
+        loss = (rng.random(K) + 20.0).astype(np.float32)
+        loss[s % K] = kept_loss                       # equal is not better (strict <)
+        before = his.x.copy()
+        his.sync(loss, want_gbest=True)
+        assert np.array_equal(his.history["row"], kept) and his.history["loss"][0] == kept_loss
+        assert np.array_equal(his.gbest, kept)
+        assert not np.array_equal(his.gbest, before[his.g])
+    # NaN never enters the history
+    his.sync(np.full(K, np.nan, np.float32))
+    assert np.array_equal(his.history["row"], kept)
+    # nothing remembered yet: the first sync takes the current best whatever its loss
+    fresh = oracle.RefSwarm(x, v, p, m_max=0.7, m_min=0.7, t_max=1, c1=1.5, c2=1.5, seed=3, history=True)
+    fresh.sync(np.full(K, np.inf, np.float32), want_gbest=True)
+    assert fresh.g == 0 and np.array_equal(fresh.gbest, x[0]) and np.array_equal(fresh.history["row"], x[0])
+    assert fresh.history["valid"][0] == 1 and np.isinf(fresh.history["loss"][0])
+    before = fresh.x.copy()
+    fresh.sync(np.array([5, 4, 3, 4, 5], np.float32), want_gbest=True)
+    assert np.array_equal(fresh.gbest, before[2]) and fresh.history["loss"][0] == 3.0
+
+
+# --------------------------------------------------------------------------
+# Synchronous SGD update (Section II-B).
+# --------------------------------------------------------------------------
+def test_ssgd_closed_forms():
+    rng = np.random.default_rng(8)
+    # K = 1: w + alpha * g, two roundings
+    w = rng.standard_normal((1, 500)).astype(np.float32)
+    g = rng.standard_normal((1, 500)).astype(np.float32)
+    w0 = w.copy()
+    oracle.ssgd(w, g, 0.25)
+    assert np.array_equal(w, w0 + np.float32(0.25) * g)
+    # small integers and a power-of-two worker count: exact
+    wi = rng.integers(-50, 50, size=(4, 333)).astype(np.float32)
+    wi[1:] = wi[0]
+    gi = rng.integers(-20, 20, size=(4, 333)).astype(np.float32)
+    expect = wi[0].astype(np.float64) + 0.5 / 4 * gi.astype(np.float64).sum(axis=0)
+    oracle.ssgd(wi, gi, 0.5)
+    assert all(np.array_equal(wi[k].astype(np.float64), expect) for k in range(4))
+    # general case against double arithmetic; sign convention is "+ alpha" as the paper writes it
+    K, n = 7, 4096
+    wg = np.tile(rng.standard_normal(n).astype(np.float32), (K, 1))
+    gg = rng.standard_normal((K, n)).astype(np.float32)
+    ref = wg[0].astype(np.float64) + (-0.01 / K) * gg.astype(np.float64).sum(axis=0)
+    mag = np.abs(wg[0]).astype(np.float64) + 0.01 / K * np.abs(gg).astype(np.float64).sum(axis=0)
+    oracle.ssgd(wg, gg, -0.01, nthreads=3)
+    assert np.all(np.abs(wg[0] - ref) <= (K + 3) * 2.0 ** -24 * mag)
+    assert all(np.array_equal(wg[0], wg[k]) for k in range(K))
+
+
+def test_ssgd_equals_averaging_of_one_local_step():
+    """Section II-B: with step = 1, averaging the workers' weights after one
+    local update w + alpha g_k is the SSGD update w + (alpha / n) sum g_k."""
+    rng = np.random.default_rng(12)
+    K, n, alpha = 8, 2000, np.float32(-0.125)
+    w = np.tile(rng.standard_normal(n).astype(np.float32), (K, 1))
+    g = rng.standard_normal((K, n)).astype(np.float32)
+    local = (w + alpha * g).astype(np.float32)
+    oracle.average(local)
+    a = w.copy()
+    oracle.ssgd(a, g, alpha)
+    scale = np.abs(w[0]) + np.abs(alpha) * np.abs(g).max(axis=0)
+    assert np.all(np.abs(local[0] - a[0]) <= 16 * 2.0 ** -24 * scale)
+
+
+def test_ssgd_respects_strides():
+    rng = np.random.default_rng(4)
+    wbuf = rng.standard_normal((3, 16)).astype(np.float32)
+    gbuf = rng.standard_normal((3, 24)).astype(np.float32)
+    keep = wbuf.copy()
+    oracle.ssgd(wbuf[:, :13], gbuf[:, :13], 0.5)
+    assert np.array_equal(wbuf[:, 13:], keep[:, 13:])
+    exp = keep[0, :13] + (np.float32(0.5) / np.float32(3)) * ((gbuf[0, :13] + gbuf[1, :13]) + gbuf[2, :13])
+    assert np.array_equal(wbuf[1, :13], exp)
