@@ -56,6 +56,7 @@ extern "C" {
 /* psops_config.flags */
 #define PSOPS_KEEP_GBEST   1u  /* keep a copy of the gBest row of each sync (+4N bytes of workspace) */
 #define PSOPS_QUADRATIC    2u  /* reserve workspace for the on-device quadratic fitness              */
+#define PSOPS_GBEST_HISTORY 4u /* gBest = best of all syncs so far instead of this sync's best (+4N bytes) */
 
 /* `which` of psops_get_weights / psops_set_weights */
 #define PSOPS_X      0         /* weights  w_i  (position of particle i)     */
@@ -67,14 +68,17 @@ typedef struct psops_ctx psops_ctx;      /* opaque */
 
 /* Hyper-parameters (Table II) and geometry of one swarm. */
 typedef struct {
-    int32_t  K;              /* particles = workers (Table I), 1..PSOPS_MAX_K              */
+    int32_t  K;              /* particles = workers (Table I) held by this context, 1..PSOPS_MAX_K */
+    int32_t  k_first;        /* swarm-wide index of row 0; 0 unless the swarm is sharded    */
     int64_t  N;              /* elements per particle, 1 .. 2^33 - 1                        */
     int64_t  ld;             /* row stride in elements, ld >= N                             */
     float    m_max, m_min;   /* Eq. 5; m_max == m_min gives a constant inertia weight       */
     int64_t  t_max;          /* Eq. 5 denominator (Max_t of Algorithm 1), >= 1              */
     float    c1, c2;         /* acceleration constants of Eq. 6                             */
     uint64_t seed;           /* Philox key                                                  */
-    uint32_t flags;          /* PSOPS_KEEP_GBEST | PSOPS_QUADRATIC                          */
+    uint32_t flags;          /* PSOPS_KEEP_GBEST | PSOPS_QUADRATIC | PSOPS_GBEST_HISTORY    */
+    int32_t  K_total;        /* particles in the whole swarm when this context holds a shard
+                                [k_first, k_first + K) of it; 0 = not sharded (K_total = K)  */
 } psops_config;
 
 /* Bytes of device workspace a context with this configuration needs
@@ -144,6 +148,50 @@ int psops_sync(psops_ctx *ctx, int64_t t_iter, float lambda);
 int psops_sync_host(psops_ctx *ctx, const float *h_x_in, int64_t h_in_ld,
                     const float *h_losses, int64_t t_iter, float lambda,
                     float *h_x_out, int64_t h_out_ld);
+
+/*
+ * Particle-sharded synchronisation: each GPU holds K of the swarm's K_total
+ * particles (psops_config.k_first / K_total) and only the best particle's
+ * weights travel -- the exchange Algorithm 3 describes as a gather of all
+ * particles reduces to an all-gather of K_total losses plus one broadcast of N
+ * floats.  Per sync, on every shard:
+ *   1. psops_set_losses with all K_total losses (the caller's all-gather);
+ *   2. psops_shard_select: Algorithm 3 and the pBest branch over the whole
+ *      swarm; *g receives the swarm-wide gBest index (waits for the stream);
+ *   3. the shard that holds particle g copies that row out (psops_get_weights)
+ *      and the caller broadcasts it into a buffer in every GPU's own memory;
+ *   4. psops_shard_update: Eq. 6 / Eq. 7 for this shard's particles with gBest
+ *      read from d_gbest_row (N floats, device pointer, 16-byte aligned on the
+ *      128-bit path).  Random draws use the swarm-wide particle index, so the
+ *      result is that of one unsharded psops_sync.
+ * psops_sync itself returns ESTATE on a sharded context.  The quadratic
+ * fitness and PSOPS_GBEST_HISTORY are not available on shards.
+ * Errors: EINVAL, EALIGN, ESTATE (no losses / update without select), ECUDA.
+ */
+int psops_shard_select(psops_ctx *ctx, int *g);
+int psops_shard_update(psops_ctx *ctx, int64_t t_iter, float lambda, const float *d_gbest_row);
+
+/*
+ * gBest from the history of all particles (the standard-PSO framework of
+ * Section II-C, step 3, in place of Algorithm 3's best-of-this-iteration):
+ * with PSOPS_GBEST_HISTORY the context remembers the best row ever selected
+ * and its loss; a sync's arg-min particle replaces it only on a strictly
+ * smaller loss (or when nothing is remembered yet), and Eq. 6 uses the
+ * remembered row.  psops_get_weights(PSOPS_GBEST) returns that row.  These two
+ * calls move the remembered loss (and, for set, the row) for checkpoint/resume.
+ */
+int psops_get_history(psops_ctx *ctx, float *gbest_loss, int *valid);
+int psops_set_history(psops_ctx *ctx, float gbest_loss, const float *gbest_row, int row_on_device);
+
+/*
+ * Synchronous SGD as the paper states it beside parameter averaging
+ * (Section II-B): w <- w + (alpha / K) sum_k grad_k, written to every row of x
+ * (the new weight is computed from row 0).  d_grad: K rows of stride grad_ld
+ * (>= N), device pointer.  fp32: gradients summed in worker order, one division
+ * alpha / K, one product, one addition.  v, pbest and the sync counter are
+ * untouched.
+ */
+int psops_ssgd(psops_ctx *ctx, const float *d_grad, int64_t grad_ld, float alpha);
 
 /*
  * Parameter averaging, the baseline the paper compares with (Section II-B,

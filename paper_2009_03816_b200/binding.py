@@ -21,7 +21,7 @@ PSOPS_EINVAL, PSOPS_EALIGN, PSOPS_ESTATE, PSOPS_ENAN = -1, -2, -3, -4
 PSOPS_EWORKSPACE, PSOPS_ECUDA, PSOPS_ENOMEM, PSOPS_ELIMIT = -5, -6, -7, -8
 PSOPS_STATIC_SCRATCH_DOUBLES = 1 << 20
 PSOPS_MAX_K = 1024
-PSOPS_KEEP_GBEST, PSOPS_QUADRATIC = 1, 2
+PSOPS_KEEP_GBEST, PSOPS_QUADRATIC, PSOPS_GBEST_HISTORY = 1, 2, 4
 PSOPS_X, PSOPS_V, PSOPS_PBEST, PSOPS_GBEST = 0, 1, 2, 3
 
 EXPORTS = [
@@ -30,15 +30,16 @@ EXPORTS = [
     "psops_sync_info", "psops_get_losses", "psops_set_quadratic",
     "psops_eval_quadratic", "psops_get_state", "psops_set_state", "psops_inertia",
     "psops_launch_count", "psops_strerror", "psops_last_error", "psops_destroy",
-    "psops_quadratic_fitness_static",
+    "psops_quadratic_fitness_static", "psops_shard_select", "psops_shard_update",
+    "psops_get_history", "psops_set_history", "psops_ssgd",
 ]
 
 
 class psops_config(ctypes.Structure):
-    _fields_ = [("K", ctypes.c_int32), ("N", ctypes.c_int64), ("ld", ctypes.c_int64),
-                ("m_max", ctypes.c_float), ("m_min", ctypes.c_float),
+    _fields_ = [("K", ctypes.c_int32), ("k_first", ctypes.c_int32), ("N", ctypes.c_int64),
+                ("ld", ctypes.c_int64), ("m_max", ctypes.c_float), ("m_min", ctypes.c_float),
                 ("t_max", ctypes.c_int64), ("c1", ctypes.c_float), ("c2", ctypes.c_float),
-                ("seed", ctypes.c_uint64), ("flags", ctypes.c_uint32)]
+                ("seed", ctypes.c_uint64), ("flags", ctypes.c_uint32), ("K_total", ctypes.c_int32)]
 
 
 class PsopsError(RuntimeError):
@@ -88,6 +89,11 @@ def load() -> ctypes.CDLL:
         "psops_strerror": (ctypes.c_char_p, [ctypes.c_int]),
         "psops_last_error": (ctypes.c_char_p, [_vp]),
         "psops_destroy": (ctypes.c_int, [_vp]),
+        "psops_shard_select": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_int)]),
+        "psops_shard_update": (ctypes.c_int, [_vp, ctypes.c_int64, ctypes.c_float, _f32p]),
+        "psops_get_history": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int)]),
+        "psops_set_history": (ctypes.c_int, [_vp, ctypes.c_float, _f32p, ctypes.c_int]),
+        "psops_ssgd": (ctypes.c_int, [_vp, _f32p, ctypes.c_int64, ctypes.c_float]),
         "psops_quadratic_fitness_static": (ctypes.c_int, [_f32p, ctypes.c_int64, ctypes.c_int32,
                                                           ctypes.c_int64, _f32p, _f32p, _f32p, _vp]),
     }
@@ -130,10 +136,11 @@ def _on_device(buf) -> int:
     return int(isinstance(buf, torch.Tensor) and buf.is_cuda)
 
 
-def make_config(K, N, ld=None, *, m_max, m_min, t_max=1, c1, c2, seed, flags=0) -> psops_config:
+def make_config(K, N, ld=None, *, m_max, m_min, t_max=1, c1, c2, seed, flags=0,
+                k_first=0, K_total=0) -> psops_config:
     ld = (int(N) + 3) // 4 * 4 if ld is None else int(ld)
-    return psops_config(int(K), int(N), ld, float(m_max), float(m_min), int(t_max),
-                        float(c1), float(c2), int(seed), int(flags))
+    return psops_config(int(K), int(k_first), int(N), ld, float(m_max), float(m_min), int(t_max),
+                        float(c1), float(c2), int(seed), int(flags), int(K_total))
 
 
 # ---- one function per C entry point --------------------------------------
@@ -168,6 +175,32 @@ def psops_sync(ctx, t_iter: int = 0, lam: float = 1.0) -> None:
 def psops_sync_host(ctx, h_x_in, h_in_ld, h_losses, t_iter, lam, h_x_out, h_out_ld) -> None:
     _check(load().psops_sync_host(ctx, _ptr(h_x_in), int(h_in_ld), _ptr(h_losses), int(t_iter),
                                   float(lam), _ptr(h_x_out), int(h_out_ld)), "psops_sync_host", ctx)
+
+
+def psops_shard_select(ctx) -> int:
+    g = ctypes.c_int(-1)
+    _check(load().psops_shard_select(ctx, ctypes.byref(g)), "psops_shard_select", ctx)
+    return int(g.value)
+
+
+def psops_shard_update(ctx, t_iter, lam, d_gbest_row) -> None:
+    _check(load().psops_shard_update(ctx, int(t_iter), float(lam), _ptr(d_gbest_row)),
+           "psops_shard_update", ctx)
+
+
+def psops_get_history(ctx):
+    loss, valid = ctypes.c_float(0.0), ctypes.c_int(0)
+    _check(load().psops_get_history(ctx, ctypes.byref(loss), ctypes.byref(valid)), "psops_get_history", ctx)
+    return float(loss.value), bool(valid.value)
+
+
+def psops_set_history(ctx, gbest_loss, gbest_row) -> None:
+    _check(load().psops_set_history(ctx, float(gbest_loss), _ptr(gbest_row), _on_device(gbest_row)),
+           "psops_set_history", ctx)
+
+
+def psops_ssgd(ctx, d_grad, grad_ld, alpha) -> None:
+    _check(load().psops_ssgd(ctx, _ptr(d_grad), int(grad_ld), float(alpha)), "psops_ssgd", ctx)
 
 
 def psops_average(ctx) -> None:
@@ -242,7 +275,7 @@ class Swarm:
     forwards to the C entry points.  No arithmetic happens here."""
 
     def __init__(self, x, v, pbest, *, N=None, m_max, m_min, t_max=1, c1, c2, seed, flags=0,
-                 stream=None):
+                 stream=None, k_first=0, K_total=0):
         for t in (x, v, pbest):
             assert t.is_cuda and t.dtype == torch.float32 and t.dim() == 2 and t.stride(1) == 1
         self.x, self.v, self.pbest = x, v, pbest
@@ -251,7 +284,8 @@ class Swarm:
         assert v.stride(0) == self.ld and pbest.stride(0) == self.ld
         self.N = int(N) if N is not None else x.shape[1]
         self.cfg = make_config(self.K, self.N, self.ld, m_max=m_max, m_min=m_min, t_max=t_max,
-                               c1=c1, c2=c2, seed=seed, flags=flags)
+                               c1=c1, c2=c2, seed=seed, flags=flags, k_first=k_first, K_total=K_total)
+        self.Kt = K_total if K_total else self.K
         nbytes = psops_workspace_bytes(self.cfg)
         if nbytes == 0:
             raise PsopsError(PSOPS_EINVAL, "psops_workspace_bytes")
@@ -266,7 +300,7 @@ class Swarm:
         if isinstance(losses, np.ndarray):
             losses = np.ascontiguousarray(losses, dtype=np.float32)
         count = losses.size if isinstance(losses, np.ndarray) else losses.numel()
-        assert count == self.K
+        assert count == self.Kt
         self._loss_ref = losses        # a device buffer is read by the next sync: keep it alive
         psops_set_losses(self.ctx, losses)
 
@@ -283,10 +317,22 @@ class Swarm:
         psops_average(self.ctx)
 
     def info(self):
-        return psops_sync_info(self.ctx, self.K)
+        return psops_sync_info(self.ctx, self.Kt)
+
+    def shard_select(self) -> int:
+        return psops_shard_select(self.ctx)
+
+    def shard_update(self, d_gbest_row, t_iter=0, lam=1.0):
+        psops_shard_update(self.ctx, t_iter, lam, d_gbest_row)
+
+    def ssgd(self, d_grad, alpha):
+        psops_ssgd(self.ctx, d_grad, d_grad.stride(0), alpha)
+
+    def history(self):
+        return psops_get_history(self.ctx)
 
     def losses(self) -> np.ndarray:
-        out = np.zeros(self.K, dtype=np.float32)
+        out = np.zeros(self.Kt, dtype=np.float32)
         psops_get_losses(self.ctx, out)
         return out
 
@@ -303,7 +349,7 @@ class Swarm:
         psops_eval_quadratic(self.ctx)
 
     def state(self):
-        return psops_get_state(self.ctx, self.K)
+        return psops_get_state(self.ctx, self.Kt)
 
     def set_state(self, step, pbest_loss):
         psops_set_state(self.ctx, step, pbest_loss)

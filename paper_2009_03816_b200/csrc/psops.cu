@@ -51,20 +51,31 @@ bool config_ok(const psops_config *c)
     if (c->t_max < 1) return false;
     if (!std::isfinite(c->m_max) || !std::isfinite(c->m_min)) return false;
     if (!std::isfinite(c->c1) || !std::isfinite(c->c2)) return false;
-    if (c->flags & ~(PSOPS_KEEP_GBEST | PSOPS_QUADRATIC)) return false;
+    if (c->flags & ~(PSOPS_KEEP_GBEST | PSOPS_QUADRATIC | PSOPS_GBEST_HISTORY)) return false;
+    // particle shard: rows [k_first, k_first + K) of a swarm of K_total particles
+    if (c->K_total == 0) {
+        if (c->k_first != 0) return false;
+    } else {
+        if (c->K_total < c->K || c->K_total > PSOPS_MAX_K) return false;
+        if (c->k_first < 0 || c->k_first + c->K > c->K_total) return false;
+        if (c->K_total > c->K && (c->flags & (PSOPS_QUADRATIC | PSOPS_GBEST_HISTORY))) return false;
+    }
     return true;
 }
+
+inline int swarm_size(const psops_config *c) { return c->K_total ? c->K_total : c->K; }
+inline bool keeps_gbest(const psops_config *c) { return (c->flags & (PSOPS_KEEP_GBEST | PSOPS_GBEST_HISTORY)) != 0; }
 
 Layout make_layout(const psops_config *c)
 {
     Layout L{};
-    const size_t kbytes = round_up(sizeof(float) * (size_t)c->K, 256);
+    const size_t kbytes = round_up(sizeof(float) * (size_t)swarm_size(c), 256);
     size_t at = 0;
     L.off_losses = at;      at += kbytes;
     L.off_pbest_loss = at;  at += kbytes;
     L.off_desc = at;        at += round_up(sizeof(SyncDesc), 256);
     L.off_gbest = at;
-    if (c->flags & PSOPS_KEEP_GBEST) at += round_up(sizeof(float) * (size_t)round_up((size_t)c->N, 4), 256);
+    if (keeps_gbest(c)) at += round_up(sizeof(float) * (size_t)round_up((size_t)c->N, 4), 256);
     L.off_partials = at;
     if (c->flags & PSOPS_QUADRATIC) {
         const size_t tiles = ((size_t)c->N + kTileElems - 1) / kTileElems;
@@ -102,6 +113,8 @@ struct psops_ctx {
     bool aligned;
     bool have_losses;
     bool synced_once;
+    bool selected;                     // psops_shard_select ran and psops_shard_update has not yet
+    int Kt;                            // particles in the whole swarm (= cfg.K unless sharded)
     uint32_t step;                     // syncs enqueued through this context (the stream's own counter is on the device)
     long long quads, tiles;
     int64_t launches;
@@ -143,9 +156,10 @@ void fill_round_keys(uint64_t seed, uint32_t (&rk)[20])
 
 int launch_select(psops_ctx *ctx)
 {
-    const int threads = (int)round_up((size_t)ctx->cfg.K, 32);
+    const int threads = (int)round_up((size_t)ctx->Kt, 32);
     psops_select_kernel<<<1, threads, 0, ctx->stream>>>(ctx->loss_src, ctx->d_losses, ctx->d_pbest_loss,
-                                                        ctx->d_desc, ctx->cfg.K);
+                                                        ctx->d_desc, ctx->Kt,
+                                                        (ctx->cfg.flags & PSOPS_GBEST_HISTORY) ? 1 : 0);
     ctx->loss_src = ctx->d_losses;     // the kernel keeps a copy there
     return check_launch(ctx, "psops_select_kernel");
 }
@@ -173,12 +187,15 @@ cudaError_t launch_update_kernel(Kernel kernel, unsigned blocks, cudaStream_t st
 }
 
 int launch_update(psops_ctx *ctx, float m, float k1, float k2, long long q_begin,
-                  long long q_end, bool fitness, cudaStream_t stream, bool after_select = false)
+                  long long q_end, bool fitness, cudaStream_t stream, bool after_select = false,
+                  const float *gbest_ext = nullptr)
 {
     if (q_end <= q_begin) return PSOPS_OK;
     UpdateParams P{};
     P.x = ctx->x; P.v = ctx->v; P.p = ctx->p;
-    P.gbest_copy = (ctx->cfg.flags & PSOPS_KEEP_GBEST) ? ctx->d_gbest : nullptr;
+    P.gbest_copy = ctx->d_gbest;
+    P.gbest_ext = gbest_ext;
+    P.i_first = ctx->cfg.k_first;
     P.dvec = ctx->dvec; P.tvec = ctx->tvec; P.partials = ctx->d_partials;
     P.desc = ctx->d_desc;
     P.ld = ctx->cfg.ld; P.N = ctx->cfg.N;
@@ -294,7 +311,9 @@ int psops_create(psops_ctx **out, const psops_config *cfg, float *d_x, float *d_
     ctx->loss_src = ctx->d_losses;
     ctx->d_pbest_loss = (float *)(ctx->ws + lay.off_pbest_loss);
     ctx->d_desc = (SyncDesc *)(ctx->ws + lay.off_desc);
-    ctx->d_gbest = (cfg->flags & PSOPS_KEEP_GBEST) ? (float *)(ctx->ws + lay.off_gbest) : nullptr;
+    ctx->d_gbest = keeps_gbest(cfg) ? (float *)(ctx->ws + lay.off_gbest) : nullptr;
+    ctx->Kt = swarm_size(cfg);
+    ctx->selected = false;
     ctx->d_partials = (cfg->flags & PSOPS_QUADRATIC) ? (double *)(ctx->ws + lay.off_partials) : nullptr;
     ctx->dvec = ctx->tvec = nullptr;
     ctx->stream = (cudaStream_t)cuda_stream;
@@ -312,8 +331,8 @@ int psops_create(psops_ctx **out, const psops_config *cfg, float *d_x, float *d_
     cudaError_t e = cudaGetDevice(&ctx->device);
     if (e == cudaSuccess) {
         // pBest_loss <- +inf (Algorithm 2 clones weights only), descriptor <- 0.
-        std::vector<float> inf((size_t)cfg->K, INFINITY);
-        e = cudaMemcpyAsync(ctx->d_pbest_loss, inf.data(), sizeof(float) * (size_t)cfg->K,
+        std::vector<float> inf((size_t)ctx->Kt, INFINITY);
+        e = cudaMemcpyAsync(ctx->d_pbest_loss, inf.data(), sizeof(float) * (size_t)ctx->Kt,
                             cudaMemcpyHostToDevice, ctx->stream);
         if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_desc, 0, sizeof(SyncDesc), ctx->stream);
         if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);   // `inf` is pageable
@@ -330,12 +349,12 @@ int psops_create(psops_ctx **out, const psops_config *cfg, float *d_x, float *d_
 int psops_set_losses(psops_ctx *ctx, const float *losses, int on_device)
 {
     if (ctx == nullptr || losses == nullptr) return PSOPS_EINVAL;
-    const size_t bytes = sizeof(float) * (size_t)ctx->cfg.K;
+    const size_t bytes = sizeof(float) * (size_t)ctx->Kt;
     if (on_device) {
         if (((uintptr_t)losses & 3u) != 0) return PSOPS_EALIGN;
         ctx->loss_src = losses;        // read (and copied) by the selection kernel of the next sync
     } else {
-        const int rc = check_host_losses(losses, ctx->cfg.K);
+        const int rc = check_host_losses(losses, ctx->Kt);
         if (rc != PSOPS_OK) return rc;
         // The source may be pageable and may be reused at once: wait for the copy.
         PSOPS_CUDA(ctx, cudaMemcpyAsync(ctx->d_losses, losses, bytes, cudaMemcpyHostToDevice, ctx->stream));
@@ -351,6 +370,7 @@ int psops_sync(psops_ctx *ctx, int64_t t_iter, float lambda)
     int rc = validate_sync_args(ctx, t_iter, lambda);
     if (rc != PSOPS_OK) return rc;
     if (!ctx->have_losses) return PSOPS_ESTATE;
+    if (ctx->Kt != ctx->cfg.K) return PSOPS_ESTATE;     // a shard needs gBest from outside: psops_shard_*
     const float m = inertia_of(&ctx->cfg, t_iter);
     const float k1 = ctx->cfg.c1 / lambda;
     const float k2 = ctx->cfg.c2 / lambda;
@@ -379,6 +399,7 @@ int psops_sync_host(psops_ctx *ctx, const float *h_x_in, int64_t h_in_ld, const 
     if (rc != PSOPS_OK) return rc;
     if (h_x_in == nullptr || h_x_out == nullptr) return PSOPS_EINVAL;
     if (h_in_ld < ctx->cfg.N || h_out_ld < ctx->cfg.N) return PSOPS_EINVAL;
+    if (ctx->Kt != ctx->cfg.K) return PSOPS_ESTATE;
     rc = check_host_losses(h_losses, ctx->cfg.K);
     if (rc != PSOPS_OK) return rc;
 
@@ -450,6 +471,82 @@ int psops_sync_host(psops_ctx *ctx, const float *h_x_in, int64_t h_in_ld, const 
     return PSOPS_OK;
 }
 
+int psops_shard_select(psops_ctx *ctx, int *g)
+{
+    if (ctx == nullptr || g == nullptr) return PSOPS_EINVAL;
+    if (!ctx->have_losses) return PSOPS_ESTATE;
+    const int rc = launch_select(ctx);
+    if (rc != PSOPS_OK) return rc;
+    PSOPS_CUDA(ctx, cudaMemcpyAsync(g, &ctx->d_desc->g, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+    PSOPS_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    ctx->selected = true;
+    ctx->synced_once = true;
+    return PSOPS_OK;
+}
+
+int psops_shard_update(psops_ctx *ctx, int64_t t_iter, float lambda, const float *d_gbest_row)
+{
+    int rc = validate_sync_args(ctx, t_iter, lambda);
+    if (rc != PSOPS_OK) return rc;
+    if (d_gbest_row == nullptr) return PSOPS_EINVAL;
+    if (((uintptr_t)d_gbest_row & 3u) || (ctx->aligned && ((uintptr_t)d_gbest_row & 15u))) return PSOPS_EALIGN;
+    if (!ctx->selected || ctx->dvec != nullptr) return PSOPS_ESTATE;
+    const float m = inertia_of(&ctx->cfg, t_iter);
+    const float k1 = ctx->cfg.c1 / lambda;
+    const float k2 = ctx->cfg.c2 / lambda;
+    rc = launch_update(ctx, m, k1, k2, 0, ctx->quads, false, ctx->stream, false, d_gbest_row);
+    if (rc != PSOPS_OK) return rc;
+    ctx->selected = false;
+    ctx->step += 1;
+    return PSOPS_OK;
+}
+
+int psops_ssgd(psops_ctx *ctx, const float *d_grad, int64_t grad_ld, float alpha)
+{
+    if (ctx == nullptr || d_grad == nullptr || grad_ld < ctx->cfg.N || !std::isfinite(alpha)) return PSOPS_EINVAL;
+    if ((uintptr_t)d_grad & 3u) return PSOPS_EALIGN;
+    const float scale = alpha / (float)ctx->cfg.K;
+    const unsigned blocks = (unsigned)((ctx->quads + kUpdateThreads - 1) / kUpdateThreads);
+    const bool aligned = ctx->aligned && (((uintptr_t)d_grad & 15u) == 0) && (grad_ld % 4 == 0);
+    if (aligned)
+        psops_ssgd_kernel<true, 8><<<blocks, kUpdateThreads, 0, ctx->stream>>>(
+            ctx->x, d_grad, ctx->cfg.ld, grad_ld, ctx->cfg.N, ctx->quads, ctx->cfg.K, scale);
+    else
+        psops_ssgd_kernel<false, 8><<<blocks, kUpdateThreads, 0, ctx->stream>>>(
+            ctx->x, d_grad, ctx->cfg.ld, grad_ld, ctx->cfg.N, ctx->quads, ctx->cfg.K, scale);
+    return check_launch(ctx, "psops_ssgd_kernel");
+}
+
+int psops_get_history(psops_ctx *ctx, float *gbest_loss, int *valid)
+{
+    if (ctx == nullptr) return PSOPS_EINVAL;
+    if (!(ctx->cfg.flags & PSOPS_GBEST_HISTORY)) return PSOPS_ESTATE;
+    SyncDesc host{};
+    PSOPS_CUDA(ctx, cudaMemcpyAsync(&host, ctx->d_desc, sizeof(SyncDesc), cudaMemcpyDeviceToHost, ctx->stream));
+    PSOPS_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    if (gbest_loss != nullptr) *gbest_loss = host.hist_loss;
+    if (valid != nullptr) *valid = host.hist_valid;
+    return PSOPS_OK;
+}
+
+int psops_set_history(psops_ctx *ctx, float gbest_loss, const float *gbest_row, int row_on_device)
+{
+    if (ctx == nullptr || gbest_row == nullptr) return PSOPS_EINVAL;
+    if (!(ctx->cfg.flags & PSOPS_GBEST_HISTORY)) return PSOPS_ESTATE;
+    if (gbest_loss != gbest_loss) return PSOPS_ENAN;
+    const int one = 1;
+    char *desc = reinterpret_cast<char *>(ctx->d_desc);
+    PSOPS_CUDA(ctx, cudaMemcpyAsync(ctx->d_gbest, gbest_row, sizeof(float) * (size_t)ctx->cfg.N,
+                                    row_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, ctx->stream));
+    PSOPS_CUDA(ctx, cudaMemcpyAsync(desc + offsetof(SyncDesc, hist_loss), &gbest_loss, sizeof(float),
+                                    cudaMemcpyHostToDevice, ctx->stream));
+    PSOPS_CUDA(ctx, cudaMemcpyAsync(desc + offsetof(SyncDesc, hist_valid), &one, sizeof(int),
+                                    cudaMemcpyHostToDevice, ctx->stream));
+    PSOPS_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    ctx->synced_once = true;           // PSOPS_GBEST can be read back
+    return PSOPS_OK;
+}
+
 int psops_average(psops_ctx *ctx)
 {
     if (ctx == nullptr) return PSOPS_EINVAL;
@@ -513,12 +610,12 @@ int psops_sync_info(psops_ctx *ctx, int *g, uint32_t *improved_words, float *pbe
     SyncDesc host{};
     PSOPS_CUDA(ctx, cudaMemcpyAsync(&host, ctx->d_desc, sizeof(SyncDesc), cudaMemcpyDeviceToHost, ctx->stream));
     if (pbest_loss != nullptr)
-        PSOPS_CUDA(ctx, cudaMemcpyAsync(pbest_loss, ctx->d_pbest_loss, sizeof(float) * (size_t)ctx->cfg.K,
+        PSOPS_CUDA(ctx, cudaMemcpyAsync(pbest_loss, ctx->d_pbest_loss, sizeof(float) * (size_t)ctx->Kt,
                                         cudaMemcpyDeviceToHost, ctx->stream));
     PSOPS_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     if (g != nullptr) *g = host.g;
     if (improved_words != nullptr)
-        std::memcpy(improved_words, host.improved, sizeof(uint32_t) * (size_t)((ctx->cfg.K + 31) / 32));
+        std::memcpy(improved_words, host.improved, sizeof(uint32_t) * (size_t)((ctx->Kt + 31) / 32));
     return PSOPS_OK;
 }
 
@@ -526,7 +623,7 @@ int psops_get_losses(psops_ctx *ctx, float *dst, int dst_on_device)
 {
     if (ctx == nullptr || dst == nullptr) return PSOPS_EINVAL;
     if (!ctx->have_losses) return PSOPS_ESTATE;
-    PSOPS_CUDA(ctx, cudaMemcpyAsync(dst, ctx->loss_src, sizeof(float) * (size_t)ctx->cfg.K,
+    PSOPS_CUDA(ctx, cudaMemcpyAsync(dst, ctx->loss_src, sizeof(float) * (size_t)ctx->Kt,
                                     dst_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost,
                                     ctx->stream));
     if (!dst_on_device) PSOPS_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
@@ -580,7 +677,7 @@ int psops_get_state(psops_ctx *ctx, uint32_t *sync_step, float *pbest_loss)
     SyncDesc host{};
     PSOPS_CUDA(ctx, cudaMemcpyAsync(&host, ctx->d_desc, sizeof(SyncDesc), cudaMemcpyDeviceToHost, ctx->stream));
     if (pbest_loss != nullptr)
-        PSOPS_CUDA(ctx, cudaMemcpyAsync(pbest_loss, ctx->d_pbest_loss, sizeof(float) * (size_t)ctx->cfg.K,
+        PSOPS_CUDA(ctx, cudaMemcpyAsync(pbest_loss, ctx->d_pbest_loss, sizeof(float) * (size_t)ctx->Kt,
                                         cudaMemcpyDeviceToHost, ctx->stream));
     PSOPS_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     ctx->step = host.next_step;
@@ -591,9 +688,9 @@ int psops_get_state(psops_ctx *ctx, uint32_t *sync_step, float *pbest_loss)
 int psops_set_state(psops_ctx *ctx, uint32_t sync_step, const float *pbest_loss)
 {
     if (ctx == nullptr || pbest_loss == nullptr) return PSOPS_EINVAL;
-    for (int i = 0; i < ctx->cfg.K; ++i)
+    for (int i = 0; i < ctx->Kt; ++i)
         if (pbest_loss[i] != pbest_loss[i]) return PSOPS_ENAN;
-    PSOPS_CUDA(ctx, cudaMemcpyAsync(ctx->d_pbest_loss, pbest_loss, sizeof(float) * (size_t)ctx->cfg.K,
+    PSOPS_CUDA(ctx, cudaMemcpyAsync(ctx->d_pbest_loss, pbest_loss, sizeof(float) * (size_t)ctx->Kt,
                                     cudaMemcpyHostToDevice, ctx->stream));
     PSOPS_CUDA(ctx, cudaMemcpyAsync(reinterpret_cast<char *>(ctx->d_desc) + offsetof(SyncDesc, next_step),
                                     &sync_step, sizeof(uint32_t), cudaMemcpyHostToDevice, ctx->stream));

@@ -26,20 +26,25 @@ struct SyncDesc {
     uint32_t step;              // sync counter s of the sync in progress (Philox counter word 2)
     uint32_t next_step;         // s of the next sync; advanced by the selection kernel so that a
                                 // captured-and-replayed sync still walks the random stream
-    int      pad;
+    int      from_kept;         // 1: gBest of this sync is the remembered row, not row g (history mode)
+    float    hist_loss;         // loss of the remembered gBest (history mode)
+    int      hist_valid;        // 0 until something is remembered
+    int      pad[2];
     uint32_t improved[PSOPS_MAX_K / 32];   // bit i: loss_i < pBest_loss_i
 };
 
 struct UpdateParams {
     float *x, *v, *p;           // K rows of stride ld
-    float *gbest_copy;          // NULL or N floats
+    float *gbest_copy;          // NULL or N floats: copy of the gBest row / the remembered gBest
+    const float *gbest_ext;     // NULL, or N floats holding gBest (a shard whose best particle lives elsewhere)
     const float *dvec, *tvec;   // quadratic fitness vectors (FITNESS only)
     double *partials;           // K x tiles tile sums (FITNESS only)
     const SyncDesc *desc;
     long long ld, N;
     long long q_begin, q_end;   // quad range of this launch (quad = 4 elements)
     long long tiles;            // ceil(N / 128)
-    int K;
+    int K;                      // rows held here
+    int i_first;                // swarm-wide index of row 0 (0 unless the swarm is sharded by particle)
     float m, k1, k2;            // inertia, c1/lambda, c2/lambda
     uint32_t rk[20];            // Philox round keys, rk[2r], rk[2r+1]
 };
@@ -182,7 +187,7 @@ __device__ __forceinline__ bool beats(const Candidate &a, const Candidate &b)
 
 __global__ void __launch_bounds__(PSOPS_MAX_K)
 psops_select_kernel(const float *loss, float *loss_keep, float *__restrict__ pbest_loss,
-                    SyncDesc *__restrict__ desc, int K)
+                    SyncDesc *__restrict__ desc, int K, int history)
 {
     // Let the update kernel that follows in the stream start its prologue; it
     // waits for this grid to finish before it reads the descriptor.
@@ -220,6 +225,19 @@ psops_select_kernel(const float *loss, float *loss_keep, float *__restrict__ pbe
         for (int w = 1; w < warps; ++w)
             if (beats(warp_best[w], c)) c = warp_best[w];
         desc->g = c.idx;
+        // Standard-PSO variant (Section II-C, step 3): gBest from the history of
+        // all particles.  The current best replaces the remembered one only on
+        // a strictly smaller loss, or when nothing is remembered yet.
+        int from_kept = 0;
+        if (history) {
+            if (!desc->hist_valid || c.loss < desc->hist_loss) {
+                desc->hist_loss = c.loss;
+                desc->hist_valid = 1;
+            } else {
+                from_kept = 1;
+            }
+        }
+        desc->from_kept = from_kept;
         const uint32_t s_now = desc->next_step;
         desc->step = s_now;
         desc->next_step = s_now + 1u;
@@ -262,14 +280,26 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
 
     // gBest = row g as it is BEFORE this sync overwrites it; this thread is the
     // only writer of these elements, so reading them first is enough.
-    const int g = P.desc->g;
+    // It comes from row g of this context, from the remembered row (history
+    // mode, when the current best did not beat it) or from a row handed in by
+    // the caller (sharded swarm).
     const uint32_t step = P.desc->step;
+    const float *gsrc = P.gbest_ext;
+    bool keep_copy = false;
+    if (gsrc == nullptr) {
+        if (P.desc->from_kept) {
+            gsrc = P.gbest_copy;
+        } else {
+            gsrc = P.x + (size_t)P.desc->g * (size_t)P.ld;
+            keep_copy = P.gbest_copy != nullptr;
+        }
+    }
     float gb[Q][4];
     float dv[Q][4], tv[Q][4];
 #pragma unroll
     for (int j = 0; j < Q; ++j) {
-        load_quad_cached<ALIGNED>(P.x + (size_t)g * (size_t)P.ld + col[j], nvalid[j], gb[j]);
-        if (P.gbest_copy != nullptr) store_quad<ALIGNED>(P.gbest_copy + col[j], nvalid[j], gb[j]);
+        load_quad_cached<ALIGNED>(gsrc + col[j], nvalid[j], gb[j]);
+        if (keep_copy) store_quad<ALIGNED>(P.gbest_copy + col[j], nvalid[j], gb[j]);
         if (FITNESS) {
             load_quad_cached<ALIGNED>(P.dvec + col[j], nvalid[j], dv[j]);
             load_quad_cached<ALIGNED>(P.tvec + col[j], nvalid[j], tv[j]);
@@ -281,17 +311,17 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
     const uint32_t pair0 = (uint32_t)(2 * q0);
 
     size_t row = 0;                          // offset of row i0
-    uint32_t impw = 0;
     for (int i0 = 0; i0 < P.K; i0 += U) {
-        if ((i0 & 31) == 0) impw = P.desc->improved[i0 >> 5];
 
         float xo[U][Q][4], vo[U][Q][4], pp[U][Q][4];
         bool imp[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int i = i0 + u;
-            imp[u] = (impw >> (i & 31)) & 1u;
+            imp[u] = false;
             if (i < P.K) {
+                const int gi = P.i_first + i;            // swarm-wide particle index
+                imp[u] = (P.desc->improved[gi >> 5] >> (gi & 31)) & 1u;
 #pragma unroll
                 for (int j = 0; j < Q; ++j) {
                     const size_t at = row + (size_t)u * (size_t)P.ld + col[j];
@@ -310,8 +340,8 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
                     const size_t at = row + (size_t)u * (size_t)P.ld + col[j];
                     const uint32_t pair = pair0 + (uint32_t)(2 * j * kUpdateThreads);
                     uint32_t ra[4], rb[4];
-                    philox4x32_10(pair, (uint32_t)i, step, 0u, P.rk, ra);
-                    philox4x32_10(pair + 1u, (uint32_t)i, step, 0u, P.rk, rb);
+                    philox4x32_10(pair, (uint32_t)(P.i_first + i), step, 0u, P.rk, ra);
+                    philox4x32_10(pair + 1u, (uint32_t)(P.i_first + i), step, 0u, P.rk, rb);
                     const uint32_t w1[4] = {ra[0], ra[2], rb[0], rb[2]};   // r1 of elements 0..3
                     const uint32_t w2[4] = {ra[1], ra[3], rb[1], rb[3]};   // r2 of elements 0..3
                     float vn[4], xn[4];
@@ -373,6 +403,40 @@ psops_average_kernel(float *__restrict__ x, long long ld, long long N, long long
 #pragma unroll
     for (int e = 0; e < 4; ++e) acc[e] = __fdiv_rn(acc[e], kf);
     for (k = 0; k < K; ++k) store_quad<ALIGNED>(x + (size_t)k * (size_t)ld + d0, nvalid, acc);
+}
+
+// ---------------------------------------------------------------------------
+// Synchronous SGD (Section II-B): w <- w + (alpha / K) sum_k grad_k, written to
+// every worker's row; the new weight is computed from row 0.
+// ---------------------------------------------------------------------------
+template <bool ALIGNED, int U>
+__global__ void __launch_bounds__(kUpdateThreads)
+psops_ssgd_kernel(float *__restrict__ w, const float *__restrict__ grad, long long ld, long long grad_ld,
+                  long long N, long long quads, int K, float scale)
+{
+    const long long q = (long long)blockIdx.x * kUpdateThreads + threadIdx.x;
+    if (q >= quads) return;
+    const long long d0 = q * 4;
+    const int nvalid = (N - d0 >= 4) ? 4 : (int)(N - d0);
+
+    float w0[4], acc[4];
+    load_quad<ALIGNED>(w + d0, nvalid, w0);
+    load_quad<ALIGNED>(grad + d0, nvalid, acc);
+    for (int k = 1; k < K; k += U) {
+        float t[U][4];
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (k + u < K) load_quad<ALIGNED>(grad + (size_t)(k + u) * (size_t)grad_ld + d0, nvalid, t[u]);
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (k + u < K) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) acc[e] = __fadd_rn(acc[e], t[u][e]);
+            }
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) w0[e] = __fadd_rn(w0[e], __fmul_rn(scale, acc[e]));
+    for (int k = 0; k < K; ++k) store_quad<ALIGNED>(w + (size_t)k * (size_t)ld + d0, nvalid, w0);
 }
 
 // ---------------------------------------------------------------------------

@@ -68,3 +68,78 @@ def test_reference_arm_prints_only_on_rank_zero():
                           "--gpus", "2", "--steps", "1", "--warmup", "0"], env=env,
                          capture_output=True, text=True, timeout=300)
     assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+# ---------------------------------------------------------------------------
+# Particle-sharded sync: collective ordering and ownership, two gloo ranks.
+# The engine behind the driver is the CPU oracle run on the full swarm by every
+# rank (tests may use the oracle); what is checked is the exchange itself.
+# ---------------------------------------------------------------------------
+SHARD_WORKER = textwrap.dedent("""
+    import json, os, sys
+    sys.path.insert(0, os.environ["PSOPS_ROOT"])
+    import numpy as np, torch
+    import torch.distributed as dist
+    import oracle
+    from paper_2009_03816_b200 import replicas, sharded
+    r = replicas.init_from_env(backend="gloo")
+    counts = [3, 2]
+    K, N = 5, 257
+    rng = np.random.default_rng(0)
+    x = rng.standard_normal((K, N)).astype(np.float32); v = np.zeros_like(x); p = x.copy()
+    full = oracle.RefSwarm(x, v, p, m_max=0.7, m_min=0.7, t_max=1, c1=1.5, c2=1.5, seed=4)
+    first = sharded.first_index(r.rank, counts)
+
+    class Engine:                       # holds only this rank's rows of the reference swarm
+        def __init__(self): self.got = None; self.log = []
+        def set_losses(self, all_losses): self.losses = all_losses.numpy().copy()
+        def shard_select(self): return oracle.argmin(self.losses)
+        def copy_row(self, row, out):
+            self.log.append(("copy", row)); out.copy_(torch.from_numpy(full.x[first + row]))
+        def shard_update(self, gbest, t, lam):
+            pre = full.x.copy()
+            full.sync(self.losses, t, lam, want_gbest=True)
+            assert np.array_equal(gbest.numpy(), full.gbest), "broadcast row is not gBest"
+            assert np.array_equal(gbest.numpy(), pre[full.g])
+
+    eng = Engine()
+    drv = sharded.ShardedSync(eng, counts, N, torch.device("cpu"))
+    gs = []
+    table = np.array([[5, 4, 3, 2, 1], [1, 2, 3, 4, 5], [2, 2, 1, 1, 3]], np.float32)
+    for s in range(3):
+        mine = torch.from_numpy(table[s, first:first + counts[r.rank]].copy())
+        gs.append(drv.sync(mine))
+        assert np.array_equal(eng.losses, table[s]), "all-gather order"
+    print(json.dumps({"rank": r.rank, "g": gs, "copies": eng.log}))
+    replicas.finish(r)
+""")
+
+
+def test_sharded_exchange_two_gloo_ranks(tmp_path):
+    import json
+    script = tmp_path / "shard_worker.py"
+    script.write_text(SHARD_WORKER)
+    port = _free_port()
+    procs = []
+    for rank in range(2):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE="2",
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), PSOPS_ROOT=ROOT,
+                   CUDA_VISIBLE_DEVICES="", OMP_NUM_THREADS="1")
+        procs.append(subprocess.Popen([sys.executable, str(script)], env=env,
+                                      stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True))
+    outs = [p.communicate(timeout=180) for p in procs]
+    for p, (out, err) in zip(procs, outs):
+        assert p.returncode == 0, err
+    res = [json.loads(o[0].strip().splitlines()[-1]) for o in outs]
+    assert res[0]["g"] == res[1]["g"] == [4, 0, 2]
+    # the owner of each gBest (and only it) copied its row out: g=4 -> rank 1 row 1, g=0 -> rank 0 row 0, g=2 -> rank 0 row 2
+    assert res[0]["copies"] == [["copy", 0], ["copy", 2]] and res[1]["copies"] == [["copy", 1]]
+
+
+def test_shard_ownership_and_traffic():
+    from paper_2009_03816_b200 import sharded
+    assert sharded.owner_of(0, [3, 2]) == (0, 0) and sharded.owner_of(3, [3, 2]) == (1, 0)
+    assert sharded.owner_of(7, [1] * 8) == (7, 0) and sharded.first_index(2, [3, 1, 4]) == 4
+    t = sharded.bytes_received_per_sync(11_173_962, [2] * 8)
+    assert t["gbest_broadcast"] == 4 * 11_173_962 and t["gather_all_particles"] == 4 * 11_173_962 * 14
+    assert t["losses_all_gather"] == 64
