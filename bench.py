@@ -31,11 +31,20 @@ UNIT = "particle-elements/s"
 FALLBACK_HBM_GBS = 6650.0           # earlier measurement on this machine, used only if no measured file
 
 # DRAM traffic of the fused update kernel from an ncu capture, per
-# particle-element, and the hash of the kernel source it was taken from.  The
-# benchmark reports null once the source has changed.
-NCU_TRAFFIC = {"source_sha256": "73b09bcfd014706686406a4faf043dd5d0d70b5a9c9fffe5a1277ea33e69777e",
-               "bytes_per_particle_element": 19.56,       # 2.503 GB / 128 M at K=32, N=4 M
+# particle-element, and the hash of the source it was taken from: everything in
+# psops_kernels.cuh up to the averaging kernel, i.e. the update kernel and all
+# it uses.  The benchmark reports null once that text has changed.
+NCU_TRAFFIC = {"source_sha256": "7f9b19c680ccd11c98bec75f37a4310eb22e6412f5796ef888a08d2c15c55bbf",
+               "bytes_per_particle_element": 19.56,       # (1.328 + 1.176) GB / 128 M at K=32, N=4 M
                "profile": "profiles/update_kernel_cfg4_n4m_full.txt"}
+KERNEL_SOURCE = os.path.join(ROOT, "paper_2009_03816_b200", "csrc", "psops_kernels.cuh")
+HASH_UNTIL = "// Kernel (c): parameter averaging"
+
+
+def update_kernel_source_sha256() -> str:
+    with open(KERNEL_SOURCE) as fh:
+        text = fh.read()
+    return hashlib.sha256(text[:text.index(HASH_UNTIL)].encode()).hexdigest()
 
 
 def parse_args():
@@ -314,12 +323,8 @@ def run_psops(args):
 
 
 def ncu_traffic(w):
-    if not NCU_TRAFFIC["source_sha256"]:
+    if not NCU_TRAFFIC["source_sha256"] or update_kernel_source_sha256() != NCU_TRAFFIC["source_sha256"]:
         return None
-    src = os.path.join(ROOT, "paper_2009_03816_b200", "csrc", "psops_kernels.cuh")
-    with open(src, "rb") as fh:
-        if hashlib.sha256(fh.read()).hexdigest() != NCU_TRAFFIC["source_sha256"]:
-            return None
     return NCU_TRAFFIC["bytes_per_particle_element"] * w.K * w.N
 
 
@@ -361,6 +366,38 @@ def graph_us_per_sync(w, dev, replays=20):
     return e0.elapsed_time(e1) * 1e3 / (replays * len(rows))
 
 
+def time_variant(w, dev, ranks, peak, flags=0, shard=None, steps=100):
+    """psops_sync with a flag set, or the select + update pair of one particle shard."""
+    import torch
+    from paper_2009_03816_b200 import binding, workloads
+    table = torch.from_numpy(workloads.losses(w)).to(dev)
+    if shard is None:
+        sw = make_swarm(w, dev, flags)
+        K_here = w.K
+
+        def step(i):
+            sw.set_losses(table[i % table.shape[0]])
+            sw.sync(0, w.lam)
+    else:
+        first, K_here = shard
+        dx, dv, dp = device_state(workloads.replace(w, K=K_here), dev)
+        sw = binding.Swarm(dx, dv, dp, N=w.N, m_max=w.omega, m_min=w.omega, c1=w.c1, c2=w.c2,
+                           seed=w.seed, k_first=first, K_total=w.K)
+        gbest = dx[0].clone()
+
+        def step(i):
+            sw.set_losses(table[i % table.shape[0]])
+            sw.shard_select()
+            sw.shard_update(gbest, 0, w.lam)
+    sec = time_region(step, steps, 5, ranks)
+    gbs = (20 * K_here * w.N + 4 * w.N) / (sec / steps) / 1e9
+    sw.close()
+    del sw
+    torch.cuda.empty_cache()
+    return {"ms_per_step": sec * 1e3 / steps, "value": K_here * w.N * steps / sec, "unit": UNIT,
+            "GBps": gbs, "frac": gbs / peak}
+
+
 def other_rows(args, dev, ranks, peak):
     """The remaining rows of the path, timed the same way (device-resident)."""
     import torch
@@ -376,14 +413,30 @@ def other_rows(args, dev, ranks, peak):
         gbs = average_bytes(w3) / (sec / 100) / 1e9
         rows["cfg3_average"] = {"ms_per_step": sec * 10, "value": w3.K * w3.N * 100 / sec, "unit": UNIT,
                                 "GBps": gbs, "frac": gbs / peak}
+        # SSGD baseline on the same rows: K gradient rows in, K weight rows out
+        grad = torch.randn((w3.K, w3.ld), device=dev, generator=torch.Generator(device=dev).manual_seed(3))
+        sec = time_region(lambda i: sw.ssgd(grad, -0.01), 100, 5, ranks)
+        gbs = (8 * w3.K * w3.N + 4 * w3.N) / (sec / 100) / 1e9
+        rows["cfg3_ssgd"] = {"ms_per_step": sec * 10, "value": w3.K * w3.N * 100 / sec, "unit": UNIT,
+                             "GBps": gbs, "frac": gbs / peak}
+        del grad
         sw.close()
         del sw
         torch.cuda.empty_cache()
+        rows["cfg3_sync_gbest_history"] = time_variant(w3, dev, ranks, peak, flags=4)
+        # what one GPU of an 8-GPU particle-sharded run does per sync: 2 of the 16 particles,
+        # gBest read from a broadcast buffer (the collectives themselves need more than one GPU)
+        rows["cfg3_shard_2_of_16"] = time_variant(w3, dev, ranks, peak, shard=(0, 2))
         w5 = workloads.CONFIGS["cfg5"]
         sw, sec, _, keep = time_sync_workload(w5, dev, 50, 5, ranks, fused_fitness=True)
         gbs = sync_bytes(w5, True) / (sec / 50) / 1e9
         rows["cfg5_sync_fused_fitness"] = {"ms_per_step": sec * 20, "value": w5.K * w5.N * 50 / sec,
                                            "unit": UNIT, "GBps": gbs, "frac": gbs / peak}
+        sec = time_region(lambda i: sw.eval_quadratic(), 50, 5, ranks)
+        tiles = (w5.N + 127) // 128
+        gbs = (4 * w5.K * w5.N + 8 * w5.N + 16 * w5.K * tiles) / (sec / 50) / 1e9
+        rows["cfg5_fitness_only"] = {"ms_per_step": sec * 20, "value": w5.K * w5.N * 50 / sec,
+                                     "unit": UNIT, "GBps": gbs, "frac": gbs / peak}
         sw.close()
         del sw, keep
         torch.cuda.empty_cache()

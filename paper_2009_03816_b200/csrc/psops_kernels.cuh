@@ -311,17 +311,25 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
     const uint32_t pair0 = (uint32_t)(2 * q0);
 
     size_t row = 0;                          // offset of row i0
+    uint32_t impw = 0;                       // improved bits of particles i0 - i0 % 32 .. +31 (local numbering)
     for (int i0 = 0; i0 < P.K; i0 += U) {
+        if ((i0 & 31) == 0) {
+            // One window of 32 bits per 32 particles, fetched ahead of the loads it
+            // steers: a per-particle fetch would sit between them and stall the
+            // in-order issue.  The window starts at swarm-wide particle i_first + i0.
+            const int base = P.i_first + i0;
+            const uint32_t lo = P.desc->improved[base >> 5];
+            const uint32_t hi = ((base >> 5) + 1 < PSOPS_MAX_K / 32) ? P.desc->improved[(base >> 5) + 1] : 0u;
+            impw = __funnelshift_r(lo, hi, base & 31);
+        }
 
         float xo[U][Q][4], vo[U][Q][4], pp[U][Q][4];
         bool imp[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int i = i0 + u;
-            imp[u] = false;
+            imp[u] = (impw >> (i & 31)) & 1u;
             if (i < P.K) {
-                const int gi = P.i_first + i;            // swarm-wide particle index
-                imp[u] = (P.desc->improved[gi >> 5] >> (gi & 31)) & 1u;
 #pragma unroll
                 for (int j = 0; j < Q; ++j) {
                     const size_t at = row + (size_t)u * (size_t)P.ld + col[j];
@@ -443,6 +451,9 @@ psops_ssgd_kernel(float *__restrict__ w, const float *__restrict__ grad, long lo
 // Kernel (d): stand-alone fitness tile sums (levels 0 and 1), and the level-2
 // finalisation shared with the fused path.
 // ---------------------------------------------------------------------------
+#ifndef PSOPS_FITNESS_ROWS
+#define PSOPS_FITNESS_ROWS 2           // rows in flight in the stand-alone fitness kernel
+#endif
 template <bool ALIGNED>
 __global__ void __launch_bounds__(kUpdateThreads)
 psops_fitness_tiles_kernel(const float *__restrict__ x, const float *__restrict__ dvec,
@@ -457,11 +468,19 @@ psops_fitness_tiles_kernel(const float *__restrict__ x, const float *__restrict_
     float dv[4], tv[4];
     load_quad_cached<ALIGNED>(dvec + d0, nvalid, dv);
     load_quad_cached<ALIGNED>(tvec + d0, nvalid, tv);
-    for (int i = 0; i < K; ++i) {
-        float xi[4];
-        load_quad<ALIGNED>(x + (size_t)i * (size_t)ld + d0, nvalid, xi);
-        const double w = fitness_tile_sum(xi, dv, tv, nvalid);
-        if ((threadIdx.x & 31) == 0) partials[(size_t)i * (size_t)tiles + (size_t)(q >> 5)] = w;
+    constexpr int U = PSOPS_FITNESS_ROWS;    // rows in flight per thread
+    for (int i0 = 0; i0 < K; i0 += U) {
+        float xi[U][4];
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (i0 + u < K) load_quad<ALIGNED>(x + (size_t)(i0 + u) * (size_t)ld + d0, nvalid, xi[u]);
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (i0 + u < K) {
+                const double w = fitness_tile_sum(xi[u], dv, tv, nvalid);
+                if ((threadIdx.x & 31) == 0)
+                    partials[(size_t)(i0 + u) * (size_t)tiles + (size_t)(q >> 5)] = w;
+            }
     }
 }
 

@@ -13,7 +13,7 @@ its columns) can be regenerated without materialising the rest.
 """
 from __future__ import annotations
 
-from dataclasses import dataclass, replace
+from dataclasses import dataclass, replace  # noqa: F401  (replace is re-exported)
 
 import numpy as np
 
