@@ -515,3 +515,41 @@ def test_device_errors_and_call_order():
         binding.psops_create(cfg, *t, ws, 16)
     assert e.value.code == binding.PSOPS_EWORKSPACE
     sw.close()
+
+
+def test_element_indices_beyond_32_bits():
+    """N just above 2^32 (the Philox counter word d >> 1 passes 2^31, element
+    offsets need 64 bits, ragged last quad).  The state is drawn on the device
+    by torch's seeded generator; the oracle follows columns sampled around the
+    interesting boundaries, read back before the first sync."""
+    gpu_util.ensure_library()
+    K, N = 2, (1 << 32) + 4099
+    ld = (N + 1023) // 1024 * 1024
+    free, _ = torch.cuda.mem_get_info()
+    if free < 3 * K * ld * 4 + (8 << 30):
+        pytest.skip("needs about 110 GB of free device memory")
+    gen = torch.Generator(device="cuda").manual_seed(2033)
+    dx = torch.empty((K, ld), dtype=torch.float32, device="cuda").normal_(0.0, 0.01, generator=gen)
+    dv = torch.empty((K, ld), dtype=torch.float32, device="cuda").normal_(0.0, 1e-3, generator=gen)
+    dp = dx.clone()
+    edges = [0, 1 << 31, (1 << 32) - 4, 1 << 32, N - 8]
+    cols = np.unique(np.concatenate(
+        [np.arange(max(0, e - 6), min(N, e + 10)) for e in edges]
+        + [np.random.default_rng(1).integers(0, N, size=500)]).astype(np.int64))
+    dcols = torch.from_numpy(cols).cuda()
+    xs, vs = dx[:, dcols].cpu().numpy(), dv[:, dcols].cpu().numpy()
+    pad_before = [t[:, N:].clone() for t in (dx, dv, dp)]
+    sw = binding.Swarm(dx, dv, dp, N=N, m_max=0.7, m_min=0.7, c1=1.5, c2=1.5, seed=0xABCDEF0123456789)
+    ref = oracle.RefSwarm(xs, vs, xs, m_max=0.7, m_min=0.7, t_max=1, c1=1.5, c2=1.5,
+                          seed=0xABCDEF0123456789, elem_index=cols)
+    for loss in ([0.9, 0.4], [0.3, 0.6], [0.35, 0.1]):
+        sw.set_losses(np.array(loss, np.float32))
+        sw.sync()
+        ref.sync(np.array(loss, np.float32))
+        g, improved, _ = sw.info()
+        assert g == ref.g and np.array_equal(improved, ref.improved)
+    for name, t, want in (("x", dx, ref.x), ("v", dv, ref.v), ("pbest", dp, ref.p)):
+        assert assert_close(t[:, dcols].cpu().numpy(), want, name) == 0
+    for t, before in zip((dx, dv, dp), pad_before):
+        assert torch.equal(t[:, N:], before)               # padding untouched
+    sw.close()
