@@ -30,6 +30,13 @@
 
 #include "psops_kernels.cuh"
 
+// Bytes of weights per pipeline stage of psops_sync_host (all K rows of one
+// element range): large enough for full PCIe efficiency, small enough that
+// filling and draining the three-stage pipeline stays a small share.
+#ifndef PSOPS_HOST_CHUNK_BYTES
+#define PSOPS_HOST_CHUNK_BYTES (64ll << 20)
+#endif
+
 namespace {
 
 // ---------------------------------------------------------------------------
@@ -424,7 +431,7 @@ int psops_sync_host(psops_ctx *ctx, const float *h_x_in, int64_t h_in_ld, const 
     if (rc != PSOPS_OK) return rc;
 
     // Element ranges of whole tiles, about 32 MiB of weights per range.
-    long long chunk_q = ((32ll << 20) / (16ll * K)) / 32 * 32;
+    long long chunk_q = (((long long)PSOPS_HOST_CHUNK_BYTES) / (16ll * K)) / 32 * 32;
     if (chunk_q < 32 * 256) chunk_q = 32 * 256;
     const long long q_total = fitness ? ctx->tiles * 32 : ctx->quads;
     size_t ev = 0;

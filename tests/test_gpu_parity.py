@@ -553,3 +553,103 @@ def test_element_indices_beyond_32_bits():
     for t, before in zip((dx, dv, dp), pad_before):
         assert torch.equal(t[:, N:], before)               # padding untouched
     sw.close()
+
+
+def test_sync_host_in_place_with_history_schedule_and_kept_gbest():
+    """Host-buffer sync where the output overwrites the input, Eq. 5 and lambda
+    vary per call, and gBest comes from the history (so some pipeline ranges
+    read the remembered row and others row g)."""
+    w = workloads.CONFIGS["cfg6"].scaled(N=1_300_003, S=6)
+    x, v, p = workloads.state(w)
+    table = workloads.losses(w)
+    table[3] = table[3] + np.float32(3.0)           # worse than anything before: history must hold
+    gpu_util.ensure_library()
+    dx, dv, dp = (gpu_util.DeviceRows(a, w.N, w.ld) for a in (x, v, p))
+    sw = binding.Swarm(dx.rows, dv.rows, dp.rows, N=w.N, m_max=w.m_max, m_min=w.m_lo, t_max=w.t_max,
+                       c1=w.c1, c2=w.c2, seed=w.seed, flags=binding.PSOPS_GBEST_HISTORY)
+    ref = oracle.RefSwarm(x[:, :w.N], v[:, :w.N], p[:, :w.N], m_max=w.m_max, m_min=w.m_lo, t_max=w.t_max,
+                          c1=w.c1, c2=w.c2, seed=w.seed, nthreads=NTHREADS, history=True)
+    h = torch.from_numpy(x.copy()).pin_memory()
+    for s in range(w.S):
+        t, lam = w.schedule(s * 97)                  # spread over the epochs
+        sw.sync_host(h, table[s], t, lam)            # in place
+        ref.sync(table[s], t, lam, want_gbest=True)
+        g, improved, pl = sw.info()
+        assert g == ref.g and np.array_equal(improved, ref.improved)
+        assert assert_close(h.numpy()[:, :w.N], ref.x, f"in-place host s={s}") == 0
+        assert np.array_equal(sw.row(PSOPS_GBEST), ref.gbest)
+    assert not np.array_equal(ref.gbest, ref.x[ref.g])          # the remembered row was in use
+    for d, want in ((dx, ref.x), (dv, ref.v), (dp, ref.p)):
+        assert assert_close(d.host(), want, "device state") == 0
+        d.check_canaries("sync_host history")
+    sw.close()
+
+
+def test_sync_host_with_fused_fitness():
+    w = workloads.CONFIGS["cfg5"].scaled(N=2_600_005, S=3)
+    pair, d, t = _quadratic_pair(w)
+    pair.gpu.eval_quadratic()
+    loss = oracle.quadratic_losses(pair.ref.x, d, t, nthreads=NTHREADS)
+    h_in = torch.from_numpy(workloads.state(w)[0]).pin_memory()
+    h_out = torch.zeros_like(h_in).pin_memory()
+    for s in range(w.S):
+        h_in[:, :w.N] = torch.from_numpy(pair.ref.x)
+        pair.gpu.sync_host(h_in, loss, 0, w.lam, h_out)
+        pair.ref.sync(loss, 0, w.lam)
+        pair.check_selection()
+        loss = oracle.quadratic_losses(pair.ref.x, d, t, nthreads=NTHREADS)
+        assert np.array_equal(pair.gpu.losses().view(np.uint32), loss.view(np.uint32))
+        assert assert_close(h_out.numpy()[:, :w.N], pair.ref.x, "host out") == 0
+    pair.check_state("sync_host fused fitness")
+    pair.check_canaries()
+    pair.close()
+
+
+def test_two_contexts_on_two_streams_do_not_interfere():
+    w = workloads.CONFIGS["cfg2"].scaled(N=400_001, S=6)
+    x, v, p = workloads.state(w)
+    table = workloads.losses(w)
+    pairs, streams = [], [torch.cuda.Stream(), torch.cuda.Stream()]
+    refs = []
+    for i, st in enumerate(streams):
+        with torch.cuda.stream(st):
+            t = [torch.from_numpy(a).cuda() for a in (x, v, p)]
+        st.synchronize()
+        pairs.append((t, binding.Swarm(*t, N=w.N, m_max=w.omega, m_min=w.omega, c1=w.c1, c2=w.c2,
+                                       seed=w.seed + i, stream=st.cuda_stream)))
+        refs.append(oracle.RefSwarm(x[:, :w.N], v[:, :w.N], p[:, :w.N], m_max=w.omega, m_min=w.omega,
+                                    t_max=1, c1=w.c1, c2=w.c2, seed=w.seed + i, nthreads=NTHREADS))
+    dt = torch.from_numpy(table).cuda()
+    torch.cuda.synchronize()
+    for s in range(w.S):                             # enqueue both without waiting in between
+        for i, (t, sw) in enumerate(pairs):
+            sw.set_losses(dt[(s + i) % w.S])
+            sw.sync()
+    torch.cuda.synchronize()
+    for i, ref in enumerate(refs):
+        for s in range(w.S):
+            ref.sync(table[(s + i) % w.S])
+        for got, want in zip(pairs[i][0], (ref.x, ref.v, ref.p)):
+            assert assert_close(got.cpu().numpy()[:, :w.N], want, f"context {i}") == 0
+        pairs[i][1].close()
+
+
+def test_ssgd_of_one_local_step_equals_averaging_on_device():
+    """Section II-B: with a sync every iteration, averaging the workers' weights
+    after one local step w + alpha g_k is the SSGD update (up to rounding)."""
+    K, N = 8, 200_003
+    rng = np.random.default_rng(3)
+    w0 = np.tile(rng.standard_normal(N).astype(np.float32), (K, 1))
+    g = rng.standard_normal((K, N)).astype(np.float32)
+    alpha = np.float32(-0.125)
+    zeros = np.zeros_like(w0)
+    a = Pair((w0 + alpha * g).astype(np.float32), zeros, zeros, N, m_max=0.7, m_min=0.7, c1=1.5, c2=1.5, seed=1)
+    b = Pair(w0, zeros, zeros, N, m_max=0.7, m_min=0.7, c1=1.5, c2=1.5, seed=1)
+    a.gpu.average()
+    dg = gpu_util.DeviceRows(g, N, (N + 3) // 4 * 4)
+    b.gpu.ssgd(dg.rows, float(alpha))
+    pa, ss = a.dx.host(), b.dx.host()
+    scale = np.abs(w0[0]) + np.abs(alpha) * np.abs(g).max(axis=0)
+    assert np.all(np.abs(pa - ss) <= 16 * 2.0 ** -24 * scale)
+    a.close()
+    b.close()
