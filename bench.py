@@ -59,6 +59,8 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=4, help="0 skips the host-buffer measurement")
     ap.add_argument("--rows", choices=["all", "none"], default="all",
                     help="also time the other rows of the path (averaging, cfg3, fused fitness)")
+    ap.add_argument("--row-steps", type=int, default=0,
+                    help="timed steps per extra row (default 100, 50 for cfg5); with --n for small captures")
     ap.add_argument("--cpu-baseline", choices=["on", "off"], default="on")
     return ap.parse_args()
 
@@ -404,43 +406,45 @@ def other_rows(args, dev, ranks, peak):
     from paper_2009_03816_b200 import workloads
     rows = {}
     try:
-        w3 = workloads.CONFIGS["cfg3"]
-        sw, sec, _, _ = time_sync_workload(w3, dev, 100, 5, ranks)
-        gbs = sync_bytes(w3) / (sec / 100) / 1e9
-        rows["cfg3_sync"] = {"ms_per_step": sec * 10, "value": w3.K * w3.N * 100 / sec, "unit": UNIT,
+        w3, w5 = workloads.CONFIGS["cfg3"], workloads.CONFIGS["cfg5"]
+        if args.n:
+            w3, w5 = w3.scaled(N=args.n), w5.scaled(N=args.n)
+        S3, S5, W = args.row_steps or 100, args.row_steps or 50, (5 if not args.row_steps else 3)
+        sw, sec, _, _ = time_sync_workload(w3, dev, S3, W, ranks)
+        gbs = sync_bytes(w3) / (sec / S3) / 1e9
+        rows["cfg3_sync"] = {"ms_per_step": sec * 1e3 / S3, "value": w3.K * w3.N * S3 / sec, "unit": UNIT,
                              "GBps": gbs, "frac": gbs / peak}
-        sec = time_region(lambda i: sw.average(), 100, 5, ranks)
-        gbs = average_bytes(w3) / (sec / 100) / 1e9
-        rows["cfg3_average"] = {"ms_per_step": sec * 10, "value": w3.K * w3.N * 100 / sec, "unit": UNIT,
+        sec = time_region(lambda i: sw.average(), S3, W, ranks)
+        gbs = average_bytes(w3) / (sec / S3) / 1e9
+        rows["cfg3_average"] = {"ms_per_step": sec * 1e3 / S3, "value": w3.K * w3.N * S3 / sec, "unit": UNIT,
                                 "GBps": gbs, "frac": gbs / peak}
         # SSGD baseline on the same rows: K gradient rows in, K weight rows out
         grad = torch.randn((w3.K, w3.ld), device=dev, generator=torch.Generator(device=dev).manual_seed(3))
-        sec = time_region(lambda i: sw.ssgd(grad, -0.01), 100, 5, ranks)
-        gbs = (8 * w3.K * w3.N + 4 * w3.N) / (sec / 100) / 1e9
-        rows["cfg3_ssgd"] = {"ms_per_step": sec * 10, "value": w3.K * w3.N * 100 / sec, "unit": UNIT,
+        sec = time_region(lambda i: sw.ssgd(grad, -0.01), S3, W, ranks)
+        gbs = (8 * w3.K * w3.N + 4 * w3.N) / (sec / S3) / 1e9
+        rows["cfg3_ssgd"] = {"ms_per_step": sec * 1e3 / S3, "value": w3.K * w3.N * S3 / sec, "unit": UNIT,
                              "GBps": gbs, "frac": gbs / peak}
         del grad
         sw.close()
         del sw
         torch.cuda.empty_cache()
-        rows["cfg3_sync_gbest_history"] = time_variant(w3, dev, ranks, peak, flags=4)
+        rows["cfg3_sync_gbest_history"] = time_variant(w3, dev, ranks, peak, flags=4, steps=S3)
         # what one GPU of an 8-GPU particle-sharded run does per sync: 2 of the 16 particles,
         # gBest read from a broadcast buffer (the collectives themselves need more than one GPU)
-        rows["cfg3_shard_2_of_16"] = time_variant(w3, dev, ranks, peak, shard=(0, 2))
-        w5 = workloads.CONFIGS["cfg5"]
-        sw, sec, _, keep = time_sync_workload(w5, dev, 50, 5, ranks, fused_fitness=True)
-        gbs = sync_bytes(w5, True) / (sec / 50) / 1e9
-        rows["cfg5_sync_fused_fitness"] = {"ms_per_step": sec * 20, "value": w5.K * w5.N * 50 / sec,
+        rows["cfg3_shard_2_of_16"] = time_variant(w3, dev, ranks, peak, shard=(0, 2), steps=S3)
+        sw, sec, _, keep = time_sync_workload(w5, dev, S5, W, ranks, fused_fitness=True)
+        gbs = sync_bytes(w5, True) / (sec / S5) / 1e9
+        rows["cfg5_sync_fused_fitness"] = {"ms_per_step": sec * 1e3 / S5, "value": w5.K * w5.N * S5 / sec,
                                            "unit": UNIT, "GBps": gbs, "frac": gbs / peak}
-        sec = time_region(lambda i: sw.eval_quadratic(), 50, 5, ranks)
+        sec = time_region(lambda i: sw.eval_quadratic(), S5, W, ranks)
         tiles = (w5.N + 127) // 128
-        gbs = (4 * w5.K * w5.N + 8 * w5.N + 16 * w5.K * tiles) / (sec / 50) / 1e9
-        rows["cfg5_fitness_only"] = {"ms_per_step": sec * 20, "value": w5.K * w5.N * 50 / sec,
+        gbs = (4 * w5.K * w5.N + 8 * w5.N + 16 * w5.K * tiles) / (sec / S5) / 1e9
+        rows["cfg5_fitness_only"] = {"ms_per_step": sec * 1e3 / S5, "value": w5.K * w5.N * S5 / sec,
                                      "unit": UNIT, "GBps": gbs, "frac": gbs / peak}
         sw.close()
         del sw, keep
         torch.cuda.empty_cache()
-        for name in ("cfg1", "cfg2"):
+        for name in (() if args.n else ("cfg1", "cfg2")):
             ws = workloads.CONFIGS[name]
             sw, sec, _, _ = time_sync_workload(ws, dev, 200, 10, ranks)
             rows[name + "_sync"] = {"us_per_step": sec / 200 * 1e6, "value": ws.K * ws.N * 200 / sec,
