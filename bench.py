@@ -34,7 +34,7 @@ FALLBACK_HBM_GBS = 6650.0           # earlier measurement on this machine, used onl
 # particle-element, and the hash of the source it was taken from: everything in
 # psops_kernels.cuh up to the averaging kernel, i.e. the update kernel and all
 # it uses.  The benchmark reports null once that text has changed.
-NCU_TRAFFIC = {"source_sha256": "7f9b19c680ccd11c98bec75f37a4310eb22e6412f5796ef888a08d2c15c55bbf",
+NCU_TRAFFIC = {"source_sha256": "ada5eebaa22a962d5e61660f02521acb7dc8cc903445cbd8c4328c8b43ec14c5",
                "bytes_per_particle_element": 19.56,       # (1.328 + 1.176) GB / 128 M at K=32, N=4 M
                "profile": "profiles/update_kernel_cfg4_n4m_full.txt"}
 KERNEL_SOURCE = os.path.join(ROOT, "paper_2009_03816_b200", "csrc", "psops_kernels.cuh")

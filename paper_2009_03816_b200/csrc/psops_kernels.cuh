@@ -144,26 +144,82 @@ __device__ __forceinline__ void store_quad(float *ptr, int nvalid, const float (
     }
 }
 
-// Level 0 and level 1 of the canonical fitness sum for one quad per lane:
-// fp32 terms dvec*(e*e), widened, added left to right, then the xor butterfly
-// over the warp.  Every lane returns the tile sum.
-__device__ __forceinline__ double fitness_tile_sum(const float (&xn)[4], const float (&dv)[4],
+// Level 0 of the canonical fitness sum for one quad: fp32 terms dvec*(e*e),
+// widened to fp64 and added left to right.
+__device__ __forceinline__ double fitness_quad_sum(const float (&xn)[4], const float (&dv)[4],
                                                    const float (&tv)[4], int nvalid)
 {
-    double q = 0.0;
+    double q;
+    if (nvalid == 4) {                       // every quad but the ragged last one: no per-element guards
+        float term[4];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        double term = 0.0;
-        if (e < nvalid) {
+        for (int e = 0; e < 4; ++e) {
             const float err = __fsub_rn(xn[e], tv[e]);
-            term = (double)__fmul_rn(dv[e], __fmul_rn(err, err));
+            term[e] = __fmul_rn(dv[e], __fmul_rn(err, err));
         }
-        q = (e == 0) ? term : __dadd_rn(q, term);
-    }
+        q = __dadd_rn(__dadd_rn(__dadd_rn((double)term[0], (double)term[1]), (double)term[2]), (double)term[3]);
+    } else {
+        q = 0.0;
 #pragma unroll
-    for (int off = 16; off >= 1; off >>= 1)
-        q = __dadd_rn(q, __shfl_xor_sync(0xffffffffu, q, off));
+        for (int e = 0; e < 4; ++e) {
+            double term = 0.0;                   // elements past the end contribute +0.0
+            if (e < nvalid) {
+                const float err = __fsub_rn(xn[e], tv[e]);
+                term = (double)__fmul_rn(dv[e], __fmul_rn(err, err));
+            }
+            q = (e == 0) ? term : __dadd_rn(q, term);
+        }
+    }
     return q;
+}
+
+// Level 1 for R rows at once (R a power of two <= 32): the xor butterfly
+// a[l] += a[l ^ off], off = 16, 8, 4, 2, 1 of every row, with the rows packed
+// into one register as the butterfly makes lanes redundant.  After the stage
+// with offset `off` lanes l and l ^ off hold the same value, so two rows can
+// share a register -- lanes with that bit clear keep the even row, lanes with
+// it set take the odd row -- and the remaining stages (smaller offsets never
+// cross that bit) reduce both at once.  Each row still goes through exactly
+// its own butterfly tree, so the result is bit-identical to R separate
+// butterflies, for R + R/2 + ... + 1 (+ what is left of the five) stages
+// instead of 5 R.  On return q[0] of lane l holds the tile sum of row
+// fitness_row_of_lane<R>(l).
+template <int R>
+__device__ __forceinline__ void fitness_tile_sums(double (&q)[R], int lane)
+{
+    static_assert(R >= 1 && R <= 32 && (R & (R - 1)) == 0, "rows per group must be a power of two");
+#pragma unroll
+    for (int s = 0; s < 5; ++s) {
+        const int off = 16 >> s;
+        const int n = (R >> s) > 0 ? (R >> s) : 1;       // registers still live at this stage
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+            if (r < n) q[r] = __dadd_rn(q[r], __shfl_xor_sync(0xffffffffu, q[r], off));
+        if (n > 1) {
+            const bool odd = (lane & off) != 0;
+#pragma unroll
+            for (int r = 0; r < R / 2; ++r)
+                if (r < n / 2) q[r] = odd ? q[2 * r + 1] : q[2 * r];
+        }
+    }
+}
+
+// Row whose tile sum lane l holds after fitness_tile_sums<R>: row bit b sits in
+// lane bit 4 - b.  All lanes that agree in those bits hold the same value.
+template <int R>
+__device__ __forceinline__ int fitness_row_of_lane(int lane)
+{
+    int row = 0;
+#pragma unroll
+    for (int b = 0; (1 << b) < R; ++b) row |= ((lane >> (4 - b)) & 1) << b;
+    return row;
+}
+
+// One lane per row writes: the one whose remaining low lane bits are zero.
+template <int R>
+__device__ __forceinline__ bool fitness_lane_writes(int lane)
+{
+    return (lane & (32 / R - 1)) == 0;
 }
 
 // ---------------------------------------------------------------------------
@@ -310,6 +366,22 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
     // 2q + 1 for elements 4q+2, 4q+3.
     const uint32_t pair0 = (uint32_t)(2 * q0);
 
+    // With the fitness fused in, the warp reduction of a batch is carried into
+    // the next iteration and runs right after that iteration's loads have been
+    // issued, so that the shuffle chain sits in the shadow of the loads.
+    double fq[Q][U];                         // level-0 fitness sums of the previous batch
+    int fq_i0 = -1;
+    const int lane = threadIdx.x & 31;
+    auto flush_fitness = [&]() {
+#pragma unroll
+        for (int j = 0; j < Q; ++j) {
+            fitness_tile_sums<U>(fq[j], lane);
+            const int i = fq_i0 + fitness_row_of_lane<U>(lane);
+            if (fitness_lane_writes<U>(lane) && active[j] && i < P.K)   // q_end is a whole number of tiles
+                P.partials[(size_t)i * (size_t)P.tiles + (col[j] >> 7)] = fq[j][0];
+        }
+    };
+
     size_t row = 0;                          // offset of row i0
     uint32_t impw = 0;                       // improved bits of particles i0 - i0 % 32 .. +31 (local numbering)
     for (int i0 = 0; i0 < P.K; i0 += U) {
@@ -338,6 +410,14 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
                     if (!imp[u]) load_quad<ALIGNED>(P.p + at, nvalid[j], pp[u][j]);
                 }
             }
+        }
+        if (FITNESS) {
+            if (fq_i0 >= 0) flush_fitness();     // previous batch, under this batch's loads
+#pragma unroll
+            for (int j = 0; j < Q; ++j)
+#pragma unroll
+                for (int u = 0; u < U; ++u) fq[j][u] = 0.0;   // rows past K carry +0.0 and are not written
+            fq_i0 = i0;
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -368,16 +448,13 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
                     store_quad<ALIGNED>(P.v + at, nvalid[j], vn);
                     store_quad<ALIGNED>(P.x + at, nvalid[j], xn);
                     if (imp[u]) store_quad<ALIGNED>(P.p + at, nvalid[j], xo[u][j]);
-                    if (FITNESS) {
-                        const double wsum = fitness_tile_sum(xn, dv[j], tv[j], nvalid[j]);
-                        if ((threadIdx.x & 31) == 0 && active[j])   // q_end is a whole number of tiles
-                            P.partials[(size_t)i * (size_t)P.tiles + (col[j] >> 7)] = wsum;
-                    }
+                    if (FITNESS) fq[j][u] = fitness_quad_sum(xn, dv[j], tv[j], nvalid[j]);
                 }
             }
         }
         row += (size_t)U * (size_t)P.ld;
     }
+    if (FITNESS && fq_i0 >= 0) flush_fitness();
 }
 
 // ---------------------------------------------------------------------------
@@ -452,7 +529,7 @@ psops_ssgd_kernel(float *__restrict__ w, const float *__restrict__ grad, long lo
 // finalisation shared with the fused path.
 // ---------------------------------------------------------------------------
 #ifndef PSOPS_FITNESS_ROWS
-#define PSOPS_FITNESS_ROWS 2           // rows in flight in the stand-alone fitness kernel
+#define PSOPS_FITNESS_ROWS 4           // rows per group in the stand-alone fitness kernel (power of two)
 #endif
 template <bool ALIGNED>
 __global__ void __launch_bounds__(kUpdateThreads)
@@ -474,13 +551,14 @@ psops_fitness_tiles_kernel(const float *__restrict__ x, const float *__restrict_
 #pragma unroll
         for (int u = 0; u < U; ++u)
             if (i0 + u < K) load_quad<ALIGNED>(x + (size_t)(i0 + u) * (size_t)ld + d0, nvalid, xi[u]);
+        double fq[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u)
-            if (i0 + u < K) {
-                const double w = fitness_tile_sum(xi[u], dv, tv, nvalid);
-                if ((threadIdx.x & 31) == 0)
-                    partials[(size_t)(i0 + u) * (size_t)tiles + (size_t)(q >> 5)] = w;
-            }
+        for (int u = 0; u < U; ++u) fq[u] = (i0 + u < K) ? fitness_quad_sum(xi[u], dv, tv, nvalid) : 0.0;
+        const int lane = threadIdx.x & 31;
+        fitness_tile_sums<U>(fq, lane);
+        const int i = i0 + fitness_row_of_lane<U>(lane);
+        if (fitness_lane_writes<U>(lane) && i < K)
+            partials[(size_t)i * (size_t)tiles + (size_t)(q >> 5)] = fq[0];
     }
 }
 
