@@ -17,6 +17,7 @@
 
 #include "psops.h"
 
+#include <cooperative_groups.h>   // thread-block clusters of the fitness finaliser
 #include <cuda_runtime.h>
 
 #include <cmath>
@@ -228,7 +229,7 @@ int launch_update(psops_ctx *ctx, float m, float k1, float k2, long long q_begin
 
 int launch_finalize(psops_ctx *ctx)
 {
-    psops_fitness_finalize_kernel<<<ctx->cfg.K, kFinalizeThreads, 0, ctx->stream>>>(
+    psops_fitness_finalize_kernel<<<dim3(kFinalizeCluster, ctx->cfg.K), kFinalizeCtaThreads, 0, ctx->stream>>>(
         ctx->d_partials, ctx->d_losses, ctx->tiles);
     ctx->loss_src = ctx->d_losses;
     return check_launch(ctx, "psops_fitness_finalize_kernel");
@@ -817,7 +818,7 @@ extern "C" int psops_quadratic_fitness_static(const float *d_x, int64_t ld, int3
         psops_fitness_tiles_kernel<false><<<blocks, kUpdateThreads, 0, stream>>>(
             d_x, d_dvec, d_tvec, tile_sums, ld, N, quads, tiles, K);
     if (cudaGetLastError() != cudaSuccess) return PSOPS_ECUDA;
-    psops_fitness_finalize_kernel<<<K, kFinalizeThreads, 0, stream>>>(tile_sums, d_loss, tiles);
+    psops_fitness_finalize_kernel<<<dim3(kFinalizeCluster, K), kFinalizeCtaThreads, 0, stream>>>(tile_sums, d_loss, tiles);
     if (cudaGetLastError() != cudaSuccess) return PSOPS_ECUDA;
     return PSOPS_OK;
 }

@@ -562,22 +562,56 @@ psops_fitness_tiles_kernel(const float *__restrict__ x, const float *__restrict_
     }
 }
 
-// One block per particle, thread tau = slot tau.
-__global__ void __launch_bounds__(kFinalizeThreads)
+// Level 2.  The 1024 slots of one particle are spread over a cluster of 8
+// thread blocks (128 slots = 4 groups of 32 each), so eight SMs stream the
+// particle's tile sums instead of one; thread tau still adds tiles tau,
+// tau + 1024, ... in increasing order (loads run ahead, the additions stay a
+// chain), each warp butterflies its group, and the 32 group sums meet in the
+// shared memory of the cluster's first block, whose first thread adds them in
+// group order.  cluster.sync() is the hardware cluster barrier.
+#ifndef PSOPS_FINALIZE_DEPTH
+#define PSOPS_FINALIZE_DEPTH 32        // tile sums in flight per thread of the finaliser
+#endif
+constexpr int kFinalizeCluster = 8;
+constexpr int kFinalizeCtaThreads = kFinalizeThreads / kFinalizeCluster;
+static_assert(kFinalizeCtaThreads % 32 == 0, "a warp is one group of 32 slots");
+
+__global__ void __cluster_dims__(kFinalizeCluster, 1, 1) __launch_bounds__(kFinalizeCtaThreads)
 psops_fitness_finalize_kernel(const double *__restrict__ partials, float *__restrict__ loss,
                               long long tiles)
 {
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
     __shared__ double group[kFinalizeThreads / 32];
-    const int i = blockIdx.x;
+    const unsigned rank = cluster.block_rank();
+    const int i = blockIdx.y;
+    const int tau = (int)rank * kFinalizeCtaThreads + (int)threadIdx.x;      // slot
     const double *row = partials + (size_t)i * (size_t)tiles;
+
     double acc = 0.0;
-    for (long long m = threadIdx.x; m < tiles; m += kFinalizeThreads) acc = __dadd_rn(acc, row[m]);
+    // Only 1024 chains per particle exist, so each thread keeps many loads in
+    // flight; the volatile asm keeps the compiler from trading them for registers.
+    constexpr int D = PSOPS_FINALIZE_DEPTH;
+    long long m = tau;
+    for (; m + (long long)(D - 1) * kFinalizeThreads < tiles; m += (long long)D * kFinalizeThreads) {
+        double v[D];
+#pragma unroll
+        for (int d = 0; d < D; ++d)
+            asm volatile("ld.global.f64 %0, [%1];" : "=d"(v[d]) : "l"(row + m + (long long)d * kFinalizeThreads));
+#pragma unroll
+        for (int d = 0; d < D; ++d) acc = __dadd_rn(acc, v[d]);
+    }
+    for (; m < tiles; m += kFinalizeThreads) acc = __dadd_rn(acc, row[m]);
+
 #pragma unroll
     for (int off = 16; off >= 1; off >>= 1)
         acc = __dadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, off));
-    if ((threadIdx.x & 31) == 0) group[threadIdx.x >> 5] = acc;
-    __syncthreads();
-    if (threadIdx.x == 0) {
+    if ((threadIdx.x & 31) == 0) {
+        double *first = cluster.map_shared_rank(group, 0);
+        first[tau >> 5] = acc;
+    }
+    cluster.sync();
+    if (rank == 0 && threadIdx.x == 0) {
         double total = group[0];
         for (int gq = 1; gq < kFinalizeThreads / 32; ++gq) total = __dadd_rn(total, group[gq]);
         loss[i] = (float)total;
