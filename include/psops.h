@@ -18,6 +18,8 @@
  *   - The library allocates no device memory.  The caller owns x, v, pbest,
  *     the workspace, dvec/tvec and the stream, and keeps them alive until
  *     psops_destroy.  The context itself is host memory owned by the library.
+ *   - A context is not thread-safe: one host thread at a time per context.
+ *     Different contexts are independent (different streams run concurrently).
  *   - Work is enqueued on the stream given at creation.  Calls that fill a
  *     host buffer wait for that stream before they return; the others do not.
  *   - Rows: particle i occupies elements [i*ld, i*ld + N) of x, v and pbest.

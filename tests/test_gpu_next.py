@@ -93,12 +93,13 @@ def test_history_gbest_matches_oracle(N, ld, offset):
     sw2.close()
 
 
-@pytest.mark.parametrize("counts", [[1, 1, 1, 1], [2, 2, 2, 2], [3, 1, 4], [8]])
+@pytest.mark.parametrize("counts", [[1, 1, 1, 1], [2, 2, 2, 2], [3, 1, 4], [8], [30, 10, 30], [33, 37]])
 def test_particle_shards_reproduce_the_unsharded_sync(counts):
     """Every shard is a context of its own with its own rows; they are driven
     one after another through the calls a multi-GPU run makes.  The result
     must be that of one unsharded swarm (the oracle)."""
-    K, N = sum(counts), 20_003
+    K = sum(counts)
+    N = 20_003 if K <= 8 else 3_001          # shards whose improved bits straddle 32-bit words
     ld = (N + 3) // 4 * 4
     x, v, p = _swarm(K, N, 5)
     gpu_util.ensure_library()
