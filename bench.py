@@ -249,15 +249,16 @@ def run_psops(args):
     _build.build_library() if ranks.local_rank == 0 else None
     replicas.barrier(ranks) if ranks.world > 1 else None
     binding.load()
-    torch.cuda.set_device(ranks.local_rank)
-    dev = torch.device("cuda", ranks.local_rank)
+    dev_index = ranks.local_rank % torch.cuda.device_count()    # replicas may share a GPU
+    torch.cuda.set_device(dev_index)
+    dev = torch.device("cuda", dev_index)
     w = workloads.CONFIGS[args.workload]
     if args.n:
         w = w.scaled(N=args.n)
     peak, peak_src = measured_peak()
     pe = w.K * w.N
 
-    sampler = ClockSampler(ranks.local_rank)
+    sampler = ClockSampler(dev_index)
     fused = w.quadratic
     sw, seconds, launches, keep = time_sync_workload(w, dev, args.steps, args.warmup, ranks, sampler, fused)
     rate, slowest = replicas.whole_job_rate(ranks, pe * args.steps, seconds)
@@ -303,7 +304,7 @@ def run_psops(args):
                    "parallelism": "replicas only"},
         "clocks": sampler.report(),
         "e2e": e2e,
-        "gpu_launches": int(launches),
+        "gpu_launches": int(replicas.sum_over_ranks(ranks, launches)),
         "roofline": {"bound": "hbm", "kernel": "psops_update_kernel", "achieved": achieved,
                      "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal_8TBs": achieved / 8000.0,

@@ -37,7 +37,9 @@ def init_from_env(backend: str | None = None) -> Ranks:
     local = int(os.environ.get("LOCAL_RANK", rank))
     os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
     if backend is None:
-        backend = "nccl" if torch.cuda.is_available() else "gloo"
+        # PSOPS_DIST_BACKEND=gloo lets independent replicas rendezvous over CPU
+        # tensors, e.g. several replicas sharing one GPU on a development box.
+        backend = os.environ.get("PSOPS_DIST_BACKEND") or ("nccl" if torch.cuda.is_available() else "gloo")
     if backend == "nccl":
         torch.cuda.set_device(local)
     dist.init_process_group(backend=backend, rank=rank, world_size=world)
