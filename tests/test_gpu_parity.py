@@ -2,6 +2,8 @@
 the same seeded inputs -- selection bit-exact, x / v / pbest within 1e-6
 relative after every sync, free-running (the GPU state is never refreshed from
 the oracle)."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -279,9 +281,11 @@ def test_cfg5_scalar_path_fused_fitness():
     pair.close()
 
 
-def test_cfg5_full_size_two_syncs():
+def test_cfg5_full_size(syncs=None):
     """Full 50 M-element vectors, fitness fused into the update; the oracle
-    runs the whole swarm on all host cores for a bounded number of syncs."""
+    runs the whole swarm on all host cores for a bounded number of syncs
+    (PSOPS_CFG5_SYNCS=200 runs the whole recipe, about 2.5 minutes)."""
+    syncs = int(os.environ.get("PSOPS_CFG5_SYNCS", "6")) if syncs is None else syncs
     w = workloads.CONFIGS["cfg5"]
     gpu_util.ensure_library()
     dev = torch.device("cuda:0")
@@ -299,8 +303,8 @@ def test_cfg5_full_size_two_syncs():
     del x, v, p
     loss = oracle.quadratic_losses(ref.x, d, t, nthreads=NTHREADS)
     cols = torch.from_numpy(workloads.sample_columns(w.N, 200_000, 5)).to(dev)
-    for s in range(2):
-        assert np.array_equal(gpu.losses().view(np.uint32), loss.view(np.uint32))
+    for s in range(syncs):
+        assert np.array_equal(gpu.losses().view(np.uint32), loss.view(np.uint32)), s
         gpu.sync(0, w.lam)
         ref.sync(loss, 0, w.lam)
         g, improved, pl = gpu.info()
