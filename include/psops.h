@@ -273,8 +273,13 @@ int psops_quadratic_fitness_static(const float *d_x, int64_t ld, int32_t K, int6
                                    const float *d_dvec, const float *d_tvec,
                                    float *d_loss, void *cuda_stream);
 
-/* Checkpoint / resume of the small state: the sync counter and pBest_loss[K]
- * (host pointers).  x, v, pbest are the caller's own tensors. */
+/* Checkpoint / resume of the small state: the sync counter (kept on the
+ * device, so both calls wait for the stream) and pBest_loss (host pointers, one
+ * float per particle of the whole swarm).  x, v, pbest are the caller's own
+ * tensors; with PSOPS_GBEST_HISTORY also move the remembered row and loss
+ * (psops_get_history / psops_set_history).  Restoring these into a new context
+ * on the same tensors continues the run bit for bit: the random stream is a
+ * function of (seed, sync counter, particle, element) only. */
 int psops_get_state(psops_ctx *ctx, uint32_t *sync_step, float *pbest_loss);
 int psops_set_state(psops_ctx *ctx, uint32_t sync_step, const float *pbest_loss);
 
