@@ -62,6 +62,9 @@ def parse_args():
     ap.add_argument("--row-steps", type=int, default=0,
                     help="timed steps per extra row (default 100, 50 for cfg5); with --n for small captures")
     ap.add_argument("--cpu-baseline", choices=["on", "off"], default="on")
+    ap.add_argument("--parallelism", choices=["replicas", "shards"], default="replicas",
+                    help="shards: ONE swarm split by particle over the ranks (all-gather of losses + "
+                         "broadcast of the best row per sync); strong scaling, not the default metric")
     return ap.parse_args()
 
 
@@ -258,6 +261,9 @@ def run_psops(args):
     peak, peak_src = measured_peak()
     pe = w.K * w.N
 
+    if args.parallelism == "shards":
+        run_shards(args, w, dev, dev_index, ranks, peak, peak_src)
+        return
     sampler = ClockSampler(dev_index)
     fused = w.quadratic
     sw, seconds, launches, keep = time_sync_workload(w, dev, args.steps, args.warmup, ranks, sampler, fused)
@@ -320,6 +326,58 @@ def run_psops(args):
             out["rows"] = other_rows(args, dev, ranks, peak)
         if args.cpu_baseline == "on":
             out["cpu_baseline"] = cpu_baseline(w)
+    if ranks.is_root:
+        print(json.dumps(out), flush=True)
+    replicas.finish(ranks)
+
+
+def run_shards(args, w, dev, dev_index, ranks, peak, peak_src):
+    """One swarm, K / world particles per rank.  Per sync every rank receives
+    4 K bytes of losses and 4 N bytes of gBest instead of the other ranks' rows."""
+    import torch
+    from paper_2009_03816_b200 import binding, replicas, sharded, workloads
+    if w.K % ranks.world or w.quadratic:
+        raise SystemExit("--parallelism shards needs K divisible by the ranks and a loss-table workload")
+    n_here = w.K // ranks.world
+    counts = [n_here] * ranks.world
+    first = sharded.first_index(ranks.rank, counts)
+    dx = torch.zeros((n_here, w.ld), dtype=torch.float32, device=dev)
+    dv = torch.zeros((n_here, w.ld), dtype=torch.float32, device=dev)
+    for r in range(n_here):
+        dx[r, :w.N] = torch.from_numpy(workloads.x_row(w, first + r)).to(dev)
+        if w.sigma_v != 0.0:
+            dv[r, :w.N] = torch.from_numpy(workloads.v_row(w, first + r)).to(dev)
+    sw = binding.Swarm(dx, dv, dx.clone(), N=w.N, m_max=w.omega, m_min=w.omega, c1=w.c1, c2=w.c2,
+                       seed=w.seed, k_first=first, K_total=w.K)
+    drv = sharded.ShardedSync(sharded.swarm_engine(sw), counts, w.N, dev)
+    table = torch.from_numpy(workloads.losses(w)).to(dev)
+    sampler = ClockSampler(dev_index)
+
+    def step(i):
+        drv.sync(table[i % table.shape[0], first:first + n_here], 0, w.lam)
+
+    seconds, launches = time_region(step, args.steps, args.warmup, ranks, sampler, counter=lambda: sw.launches)
+    slowest = replicas.max_over_ranks(ranks, seconds)
+    bytes_here = 20 * n_here * w.N + 4 * w.N
+    achieved = bytes_here / (seconds / args.steps) / 1e9
+    out = {
+        "metric": METRIC, "value": w.K * w.N * args.steps / slowest, "unit": UNIT, "n_gpus": ranks.world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": slowest * 1e3 / args.steps,
+        "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": f"{w.name}: K={w.K} particles x N={w.N} fp32 ({w.note}), one swarm sharded by particle",
+                   "K": w.K, "N": w.N, "ld": w.ld, "particles_per_rank": n_here,
+                   "parallelism": f"particle shards x{ranks.world}",
+                   "exchange_bytes_per_rank_per_sync": sharded.bytes_received_per_sync(w.N, counts)},
+        "clocks": sampler.report(), "e2e": None,
+        "gpu_launches": int(replicas.sum_over_ranks(ranks, launches)),
+        "roofline": {"bound": "hbm", "kernel": "psops_update_kernel", "achieved": achieved, "peak": peak,
+                     "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
+                     "bytes_per_launch": bytes_here, "traffic": None,
+                     "note": "duration = timed region / steps: collectives, selection (with its host read of g) "
+                             "and update of this rank's particles"},
+    }
+    sw.close()
     if ranks.is_root:
         print(json.dumps(out), flush=True)
     replicas.finish(ranks)
