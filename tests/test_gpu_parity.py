@@ -657,3 +657,33 @@ def test_ssgd_of_one_local_step_equals_averaging_on_device():
     assert np.all(np.abs(pa - ss) <= 16 * 2.0 ** -24 * scale)
     a.close()
     b.close()
+
+
+def test_subnormal_overflow_and_nan_values_follow_ieee_on_both_sides():
+    """No flush-to-zero anywhere: subnormal weights and velocities stay
+    subnormal; overflow gives inf and inf - inf gives NaN in the same elements
+    on the GPU and in the oracle."""
+    K, N = 4, 4099
+    rng = np.random.default_rng(77)
+    x = (rng.standard_normal((K, N)) * 1e-39).astype(np.float32)            # subnormal
+    v = (rng.standard_normal((K, N)) * 3e-42).astype(np.float32)
+    p = (rng.standard_normal((K, N)) * 1e-38).astype(np.float32)
+    x[:, 100:200] = (rng.uniform(-1, 1, (K, 100)) * 3e38).astype(np.float32)   # overflows in Eq. 6/7
+    v[:, 100:200] = (rng.uniform(-1, 1, (K, 100)) * 3e38).astype(np.float32)
+    x[1, 300] = np.inf
+    x[2, 301] = -np.inf
+    p[3, 302] = np.nan
+    assert np.any((np.abs(x) > 0) & (np.abs(x) < 1.17e-38))
+    pair = Pair(x, v, p, N, m_max=0.9, m_min=0.9, c1=2.0, c2=2.0, seed=5)
+    with np.errstate(all="ignore"):
+        for s, loss in enumerate(([4, 3, 2, 1], [1, 2, 3, 4], [2, 1, 2, 1])):
+            pair.sync(np.array(loss, np.float32))
+            pair.check_selection()
+            for d, want, name in ((pair.dx, pair.ref.x, "x"), (pair.dv, pair.ref.v, "v"), (pair.dp, pair.ref.p, "p")):
+                got = d.host()
+                assert np.array_equal(np.isnan(got), np.isnan(want)), name
+                ok = ~np.isnan(want)
+                assert np.array_equal(got[ok], want[ok]), f"{name} s={s}"      # values (+0 == -0)
+    sub = (np.abs(pair.ref.v) > 0) & (np.abs(pair.ref.v) < 1.17e-38)
+    assert sub.any() and np.isinf(pair.ref.x).any() and np.isnan(pair.ref.x).any()
+    pair.close()
