@@ -18,6 +18,8 @@
  *   - The library allocates no device memory.  The caller owns x, v, pbest,
  *     the workspace, dvec/tvec and the stream, and keeps them alive until
  *     psops_destroy.  The context itself is host memory owned by the library.
+ *   - A context belongs to the GPU that was current in psops_create; later
+ *     calls switch to that GPU for their duration if another one is current.
  *   - A context is not thread-safe: one host thread at a time per context.
  *     Different contexts are independent (different streams run concurrently).
  *   - Work is enqueued on the stream given at creation.  Calls that fill a

@@ -151,6 +151,29 @@ int check_launch(psops_ctx *ctx, const char *what)
     return PSOPS_OK;
 }
 
+// Work of a context belongs to the device that was current at psops_create.
+// Entry points that touch the device switch to it if the caller has another
+// one current, and switch back on return.
+class DeviceGuard {
+public:
+    explicit DeviceGuard(const psops_ctx *ctx) : previous_(-1)
+    {
+        int now = -1;
+        if (ctx != nullptr && cudaGetDevice(&now) == cudaSuccess && now != ctx->device &&
+            cudaSetDevice(ctx->device) == cudaSuccess)
+            previous_ = now;
+    }
+    ~DeviceGuard()
+    {
+        if (previous_ >= 0) cudaSetDevice(previous_);
+    }
+    DeviceGuard(const DeviceGuard &) = delete;
+    DeviceGuard &operator=(const DeviceGuard &) = delete;
+
+private:
+    int previous_;
+};
+
 void fill_round_keys(uint64_t seed, uint32_t (&rk)[20])
 {
     uint32_t k0 = (uint32_t)(seed & 0xffffffffu), k1 = (uint32_t)(seed >> 32);
@@ -356,6 +379,7 @@ int psops_create(psops_ctx **out, const psops_config *cfg, float *d_x, float *d_
 
 int psops_set_losses(psops_ctx *ctx, const float *losses, int on_device)
 {
+    DeviceGuard device_guard(ctx);
     if (ctx == nullptr || losses == nullptr) return PSOPS_EINVAL;
     const size_t bytes = sizeof(float) * (size_t)ctx->Kt;
     if (on_device) {
@@ -375,6 +399,7 @@ int psops_set_losses(psops_ctx *ctx, const float *losses, int on_device)
 
 int psops_sync(psops_ctx *ctx, int64_t t_iter, float lambda)
 {
+    DeviceGuard device_guard(ctx);
     int rc = validate_sync_args(ctx, t_iter, lambda);
     if (rc != PSOPS_OK) return rc;
     if (!ctx->have_losses) return PSOPS_ESTATE;
@@ -403,6 +428,7 @@ int psops_sync(psops_ctx *ctx, int64_t t_iter, float lambda)
 int psops_sync_host(psops_ctx *ctx, const float *h_x_in, int64_t h_in_ld, const float *h_losses,
                     int64_t t_iter, float lambda, float *h_x_out, int64_t h_out_ld)
 {
+    DeviceGuard device_guard(ctx);
     int rc = validate_sync_args(ctx, t_iter, lambda);
     if (rc != PSOPS_OK) return rc;
     if (h_x_in == nullptr || h_x_out == nullptr) return PSOPS_EINVAL;
@@ -481,6 +507,7 @@ int psops_sync_host(psops_ctx *ctx, const float *h_x_in, int64_t h_in_ld, const 
 
 int psops_shard_select(psops_ctx *ctx, int *g)
 {
+    DeviceGuard device_guard(ctx);
     if (ctx == nullptr || g == nullptr) return PSOPS_EINVAL;
     if (!ctx->have_losses) return PSOPS_ESTATE;
     const int rc = launch_select(ctx);
@@ -494,6 +521,7 @@ int psops_shard_select(psops_ctx *ctx, int *g)
 
 int psops_shard_update(psops_ctx *ctx, int64_t t_iter, float lambda, const float *d_gbest_row)
 {
+    DeviceGuard device_guard(ctx);
     int rc = validate_sync_args(ctx, t_iter, lambda);
     if (rc != PSOPS_OK) return rc;
     if (d_gbest_row == nullptr) return PSOPS_EINVAL;
@@ -511,6 +539,7 @@ int psops_shard_update(psops_ctx *ctx, int64_t t_iter, float lambda, const float
 
 int psops_ssgd(psops_ctx *ctx, const float *d_grad, int64_t grad_ld, float alpha)
 {
+    DeviceGuard device_guard(ctx);
     if (ctx == nullptr || d_grad == nullptr || grad_ld < ctx->cfg.N || !std::isfinite(alpha)) return PSOPS_EINVAL;
     if ((uintptr_t)d_grad & 3u) return PSOPS_EALIGN;
     const float scale = alpha / (float)ctx->cfg.K;
@@ -527,6 +556,7 @@ int psops_ssgd(psops_ctx *ctx, const float *d_grad, int64_t grad_ld, float alpha
 
 int psops_get_history(psops_ctx *ctx, float *gbest_loss, int *valid)
 {
+    DeviceGuard device_guard(ctx);
     if (ctx == nullptr) return PSOPS_EINVAL;
     if (!(ctx->cfg.flags & PSOPS_GBEST_HISTORY)) return PSOPS_ESTATE;
     SyncDesc host{};
@@ -539,6 +569,7 @@ int psops_get_history(psops_ctx *ctx, float *gbest_loss, int *valid)
 
 int psops_set_history(psops_ctx *ctx, float gbest_loss, const float *gbest_row, int row_on_device)
 {
+    DeviceGuard device_guard(ctx);
     if (ctx == nullptr || gbest_row == nullptr) return PSOPS_EINVAL;
     if (!(ctx->cfg.flags & PSOPS_GBEST_HISTORY)) return PSOPS_ESTATE;
     if (gbest_loss != gbest_loss) return PSOPS_ENAN;
@@ -557,6 +588,7 @@ int psops_set_history(psops_ctx *ctx, float gbest_loss, const float *gbest_row, 
 
 int psops_average(psops_ctx *ctx)
 {
+    DeviceGuard device_guard(ctx);
     if (ctx == nullptr) return PSOPS_EINVAL;
     const unsigned blocks = (unsigned)((ctx->quads + kUpdateThreads - 1) / kUpdateThreads);
     if (ctx->aligned)
@@ -584,6 +616,7 @@ static int row_pointer(psops_ctx *ctx, int which, int k, float **row)
 
 int psops_get_weights(psops_ctx *ctx, int which, int k, float *dst, int dst_on_device)
 {
+    DeviceGuard device_guard(ctx);
     if (ctx == nullptr || dst == nullptr) return PSOPS_EINVAL;
     float *row = nullptr;
     const int rc = row_pointer(ctx, which, k, &row);
@@ -598,6 +631,7 @@ int psops_get_weights(psops_ctx *ctx, int which, int k, float *dst, int dst_on_d
 
 int psops_set_weights(psops_ctx *ctx, int which, int k, const float *src, int src_on_device)
 {
+    DeviceGuard device_guard(ctx);
     if (ctx == nullptr || src == nullptr) return PSOPS_EINVAL;
     if (which == PSOPS_GBEST) return PSOPS_EINVAL;
     float *row = nullptr;
@@ -613,6 +647,7 @@ int psops_set_weights(psops_ctx *ctx, int which, int k, const float *src, int sr
 
 int psops_sync_info(psops_ctx *ctx, int *g, uint32_t *improved_words, float *pbest_loss)
 {
+    DeviceGuard device_guard(ctx);
     if (ctx == nullptr) return PSOPS_EINVAL;
     if (!ctx->synced_once) return PSOPS_ESTATE;
     SyncDesc host{};
@@ -629,6 +664,7 @@ int psops_sync_info(psops_ctx *ctx, int *g, uint32_t *improved_words, float *pbe
 
 int psops_get_losses(psops_ctx *ctx, float *dst, int dst_on_device)
 {
+    DeviceGuard device_guard(ctx);
     if (ctx == nullptr || dst == nullptr) return PSOPS_EINVAL;
     if (!ctx->have_losses) return PSOPS_ESTATE;
     PSOPS_CUDA(ctx, cudaMemcpyAsync(dst, ctx->loss_src, sizeof(float) * (size_t)ctx->Kt,
@@ -657,6 +693,7 @@ int psops_set_quadratic(psops_ctx *ctx, const float *d_dvec, const float *d_tvec
 
 int psops_eval_quadratic(psops_ctx *ctx)
 {
+    DeviceGuard device_guard(ctx);
     if (ctx == nullptr) return PSOPS_EINVAL;
     if (ctx->dvec == nullptr) return PSOPS_ESTATE;
     const long long threads = ctx->tiles * 32;
@@ -679,6 +716,7 @@ int psops_eval_quadratic(psops_ctx *ctx)
 
 int psops_get_state(psops_ctx *ctx, uint32_t *sync_step, float *pbest_loss)
 {
+    DeviceGuard device_guard(ctx);
     if (ctx == nullptr) return PSOPS_EINVAL;
     // The counter lives on the device (a replayed graph advances it without
     // the host taking part), so read it from there.
@@ -695,6 +733,7 @@ int psops_get_state(psops_ctx *ctx, uint32_t *sync_step, float *pbest_loss)
 
 int psops_set_state(psops_ctx *ctx, uint32_t sync_step, const float *pbest_loss)
 {
+    DeviceGuard device_guard(ctx);
     if (ctx == nullptr || pbest_loss == nullptr) return PSOPS_EINVAL;
     for (int i = 0; i < ctx->Kt; ++i)
         if (pbest_loss[i] != pbest_loss[i]) return PSOPS_ENAN;
@@ -729,6 +768,7 @@ const char *psops_last_error(const psops_ctx *ctx) { return ctx ? ctx->err : "";
 
 int psops_destroy(psops_ctx *ctx)
 {
+    DeviceGuard device_guard(ctx);
     if (ctx == nullptr) return PSOPS_EINVAL;
     int rc = PSOPS_OK;
     if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) rc = PSOPS_ECUDA;
