@@ -35,7 +35,7 @@ FALLBACK_HBM_GBS = 6650.0           # earlier measurement on this machine, used onl
 # psops_kernels.cuh up to the averaging kernel, i.e. the update kernel and all
 # it uses.  The benchmark reports null once that text has changed.
 NCU_TRAFFIC = {"source_sha256": "ada5eebaa22a962d5e61660f02521acb7dc8cc903445cbd8c4328c8b43ec14c5",
-               "bytes_per_particle_element": 19.56,       # (1.328 + 1.176) GB / 128 M at K=32, N=4 M
+               "bytes_per_particle_element": 19.93,       # 16.30 GB / 817.8 M: full-size cfg4 launches, 1-pass counters
                "profile": "profiles/update_kernel_cfg4_n4m_full.txt"}
 KERNEL_SOURCE = os.path.join(ROOT, "paper_2009_03816_b200", "csrc", "psops_kernels.cuh")
 HASH_UNTIL = "// Kernel (c): parameter averaging"
