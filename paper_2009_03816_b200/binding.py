@@ -32,6 +32,7 @@ EXPORTS = [
     "psops_launch_count", "psops_strerror", "psops_last_error", "psops_destroy",
     "psops_quadratic_fitness_static", "psops_shard_select", "psops_shard_update",
     "psops_get_history", "psops_set_history", "psops_ssgd",
+    "psops_host_register", "psops_host_unregister",
 ]
 
 
@@ -94,6 +95,8 @@ def load() -> ctypes.CDLL:
         "psops_get_history": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int)]),
         "psops_set_history": (ctypes.c_int, [_vp, ctypes.c_float, _f32p, ctypes.c_int]),
         "psops_ssgd": (ctypes.c_int, [_vp, _f32p, ctypes.c_int64, ctypes.c_float]),
+        "psops_host_register": (ctypes.c_int, [_vp, ctypes.c_size_t]),
+        "psops_host_unregister": (ctypes.c_int, [_vp]),
         "psops_quadratic_fitness_static": (ctypes.c_int, [_f32p, ctypes.c_int64, ctypes.c_int32,
                                                           ctypes.c_int64, _f32p, _f32p, _f32p, _vp]),
     }
@@ -201,6 +204,16 @@ def psops_set_history(ctx, gbest_loss, gbest_row) -> None:
 
 def psops_ssgd(ctx, d_grad, grad_ld, alpha) -> None:
     _check(load().psops_ssgd(ctx, _ptr(d_grad), int(grad_ld), float(alpha)), "psops_ssgd", ctx)
+
+
+def psops_host_register(buf) -> None:
+    """Pin a host buffer (numpy array or CPU tensor) in place for psops_sync_host."""
+    nbytes = buf.nbytes if isinstance(buf, np.ndarray) else buf.numel() * buf.element_size()
+    _check(load().psops_host_register(_ptr(buf), int(nbytes)), "psops_host_register")
+
+
+def psops_host_unregister(buf) -> None:
+    _check(load().psops_host_unregister(_ptr(buf)), "psops_host_unregister")
 
 
 def psops_average(ctx) -> None:

@@ -586,6 +586,31 @@ int psops_set_history(psops_ctx *ctx, float gbest_loss, const float *gbest_row, 
     return PSOPS_OK;
 }
 
+int psops_host_register(void *host_ptr, size_t bytes)
+{
+    if (host_ptr == nullptr || bytes == 0) return PSOPS_EINVAL;
+    const cudaError_t e = cudaHostRegister(host_ptr, bytes, cudaHostRegisterDefault);
+    if (e == cudaErrorHostMemoryAlreadyRegistered) {
+        (void)cudaGetLastError();
+        return PSOPS_OK;
+    }
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        return PSOPS_ECUDA;
+    }
+    return PSOPS_OK;
+}
+
+int psops_host_unregister(void *host_ptr)
+{
+    if (host_ptr == nullptr) return PSOPS_EINVAL;
+    if (cudaHostUnregister(host_ptr) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return PSOPS_ECUDA;
+    }
+    return PSOPS_OK;
+}
+
 int psops_average(psops_ctx *ctx)
 {
     DeviceGuard device_guard(ctx);

@@ -687,3 +687,24 @@ def test_subnormal_overflow_and_nan_values_follow_ieee_on_both_sides():
     sub = (np.abs(pair.ref.v) > 0) & (np.abs(pair.ref.v) < 1.17e-38)
     assert sub.any() and np.isinf(pair.ref.x).any() and np.isnan(pair.ref.x).any()
     pair.close()
+
+
+def test_host_register_pins_a_numpy_buffer_for_sync_host():
+    w = workloads.CONFIGS["cfg2"].scaled(N=1_500_003, S=2)
+    x, v, p = workloads.state(w)
+    table = workloads.losses(w)
+    pair = Pair(x, v, p, w.N, ld=w.ld, m_max=w.omega, m_min=w.omega, c1=w.c1, c2=w.c2, seed=w.seed)
+    h = x.copy()                                        # plain numpy memory
+    binding.psops_host_register(h)
+    binding.psops_host_register(h)                      # twice is fine
+    assert torch.from_numpy(h).is_pinned()
+    try:
+        for s in range(w.S):
+            pair.gpu.sync_host(h, table[s], 0, w.lam)   # in place
+            pair.ref.sync(table[s], 0, w.lam)
+            assert assert_close(h[:, :w.N], pair.ref.x, "registered host buffer") == 0
+    finally:
+        binding.psops_host_unregister(h)
+    with pytest.raises(binding.PsopsError):
+        binding.psops_host_unregister(h)                # no longer registered
+    pair.close()

@@ -96,6 +96,12 @@ def test_static_fitness_validates_before_touching_cuda(lib):
     assert f(fake, n, 2, n, fake, fake, fake, None) == binding.PSOPS_ELIMIT         # 2 * tiles > limit
 
 
+def test_host_register_rejects_null(lib):
+    assert lib.psops_host_register(None, 16) == binding.PSOPS_EINVAL
+    assert lib.psops_host_register(0x10000, 0) == binding.PSOPS_EINVAL
+    assert lib.psops_host_unregister(None) == binding.PSOPS_EINVAL
+
+
 def test_strerror_is_distinct_per_code(lib):
     texts = {lib.psops_strerror(c).decode() for c in range(0, -9, -1)}
     assert len(texts) == 9
