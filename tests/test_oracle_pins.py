@@ -638,3 +638,21 @@ def test_ssgd_respects_strides():
     assert np.array_equal(wbuf[:, 13:], keep[:, 13:])
     exp = keep[0, :13] + (np.float32(0.5) / np.float32(3)) * ((gbuf[0, :13] + gbuf[1, :13]) + gbuf[2, :13])
     assert np.array_equal(wbuf[1, :13], exp)
+
+
+def test_update_is_exactly_homogeneous_under_power_of_two_scaling():
+    """Eq. 6 / Eq. 7 are linear in (w, v, pBest): scaling the whole state by
+    2^k scales every intermediate exactly, so the result scales bit for bit."""
+    K, n = 4, 515
+    x, v, p = _random_swarm(K, n, 29)
+    loss = np.array([0.4, 0.9, 0.3, 0.8], np.float32)
+    outs = []
+    for k in (0, 7, -9):
+        f = np.float32(2.0 ** k)
+        sw = oracle.RefSwarm(x * f, v * f, p * f, m_max=0.9, m_min=0.3, t_max=10, c1=0.2, c2=0.9, seed=12)
+        sw.sync(loss, t=4, lam=3.0)
+        sw.sync(loss[::-1].copy(), t=5, lam=3.0)
+        outs.append((sw.x / f, sw.v / f, sw.p / f))
+    for a in outs[1:]:
+        for got, want in zip(a, outs[0]):
+            assert np.array_equal(got, want)
