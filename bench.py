@@ -441,7 +441,7 @@ def time_variant(w, dev, ranks, peak, flags=0, shard=None, steps=100):
             sw.sync(0, w.lam)
     else:
         first, K_here = shard
-        dx, dv, dp = device_state(workloads.replace(w, K=K_here), dev)
+        dx, dv, dp = device_state(w.with_particles(K_here), dev)
         sw = binding.Swarm(dx, dv, dp, N=w.N, m_max=w.omega, m_min=w.omega, c1=w.c1, c2=w.c2,
                            seed=w.seed, k_first=first, K_total=w.K)
         gbest = dx[0].clone()

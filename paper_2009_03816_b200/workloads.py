@@ -13,7 +13,7 @@ its columns) can be regenerated without materialising the rest.
 """
 from __future__ import annotations
 
-from dataclasses import dataclass, replace  # noqa: F401  (replace is re-exported)
+from dataclasses import dataclass, replace
 
 import numpy as np
 
@@ -71,6 +71,10 @@ class Workload:
             return 0, self.lam
         t = (s + 1) * self.sync_period
         return t, float(min(self.epochs, 1 + (t - 1) // self.iters_per_epoch))
+
+    def with_particles(self, K: int) -> "Workload":
+        """Same recipe with another number of rows (e.g. the rows one shard holds)."""
+        return replace(self, K=int(K))
 
     def scaled(self, N: int, S: int | None = None) -> "Workload":
         """Same recipe at another vector length (parity cases that a CPU
