@@ -104,8 +104,8 @@ int psops_create(psops_ctx **out, const psops_config *cfg,
                  void *d_workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
- * Hand in the K current training losses (the fitness of Table I; lower is
- * better).  on_device == 0: host pointer, checked for NaN (ENAN) and copied
+ * Hand in the current training losses of the whole swarm (the fitness of
+ * Table I; lower is better): K floats, K_total on a shard.  on_device == 0: host pointer, checked for NaN (ENAN) and copied
  * before the call returns to the stream (the buffer may be reused at once).
  * on_device != 0: device pointer (4-byte aligned), not inspected and not
  * copied now: the selection kernel of the next psops_sync reads it on the
