@@ -31,8 +31,10 @@
  *
  * Pins (see tests): Philox known-answer vectors and an independent
  * big-integer implementation; hand-worked K=2 and K=3 updates; exact
- * identities; brute-force selection; closed forms for the schedule, the
- * average and the fitness.  No function in this file is "parity unpinned".
+ * identities; brute-force selection; closed forms for the schedule and the
+ * average; for the fitness, closed forms plus hand-worked cancellation cases
+ * in which every level of the summation order and the rounding of a term
+ * change the fp32 result.  No function in this file is "parity unpinned".
  */
 #include <math.h>
 #include <stdint.h>

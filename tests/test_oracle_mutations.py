@@ -13,6 +13,17 @@ from conftest import ROOT
 SRC = os.path.join(ROOT, "oracle", "psops_ref.c")
 CFLAGS = ["-O2", "-std=c11", "-ffp-contract=off", "-fno-fast-math", "-fopenmp", "-fPIC", "-shared"]
 
+# multi-line passages of the oracle that several mutants rewrite
+_QUAD_L2R = ("double a = quad_term(x, dvec, tvec, j, N);\n"
+             "            a = a + quad_term(x, dvec, tvec, j + 1, N);\n"
+             "            a = a + quad_term(x, dvec, tvec, j + 2, N);\n"
+             "            a = a + quad_term(x, dvec, tvec, j + 3, N);")
+_GROUPS_IN_ORDER = ("for (int grp = 0; grp < 32; ++grp) {\n"
+                    "        double a[32];\n"
+                    "        for (int l = 0; l < 32; ++l) a[l] = slot[grp * 32 + l];\n"
+                    "        double gsum = butterfly32(a);\n"
+                    "        total = (grp == 0) ? gsum : total + gsum;")
+
 MUTANTS = [
     ("philox multiplier", "0xD2511F53u", "0xD2511F52u"),
     ("philox key increment", "0xBB67AE85u", "0xBB67AE86u"),
@@ -71,6 +82,38 @@ MUTANTS = [
     ("fitness drops the last element of a quad", "a = a + quad_term(x, dvec, tvec, j + 3, N);", ""),
     ("fitness drops tiles beyond the slots", "slot[mt % 1024] = slot[mt % 1024] + butterfly32(q);",
      "if (mt < 1024) slot[mt] = slot[mt] + butterfly32(q);"),
+    # summation order and term rounding of the fitness (the hand-worked cancellation cases)
+    ("fitness butterfly stages 1 -> 16", "for (int off = 16; off >= 1; off >>= 1) {",
+     "for (int off = 1; off <= 16; off <<= 1) {"),
+    ("fitness quad added right to left", _QUAD_L2R,
+     "double a = quad_term(x, dvec, tvec, j + 3, N);\n"
+     "            a = a + quad_term(x, dvec, tvec, j + 2, N);\n"
+     "            a = a + quad_term(x, dvec, tvec, j + 1, N);\n"
+     "            a = a + quad_term(x, dvec, tvec, j, N);"),
+    ("fitness quad added pairwise", _QUAD_L2R,
+     "double a = (quad_term(x, dvec, tvec, j, N) + quad_term(x, dvec, tvec, j + 1, N))\n"
+     "                   + (quad_term(x, dvec, tvec, j + 2, N) + quad_term(x, dvec, tvec, j + 3, N));"),
+    ("fitness quad accumulated in fp32", "double a = quad_term(x, dvec, tvec, j, N);",
+     "float a = (float)quad_term(x, dvec, tvec, j, N);"),
+    ("fitness tile quads added one after another", "slot[mt % 1024] = slot[mt % 1024] + butterfly32(q);",
+     "{ double ts = q[0]; for (int l = 1; l < 32; ++l) ts = ts + q[l]; slot[mt % 1024] = slot[mt % 1024] + ts; }"),
+    ("fitness 512 slots", "slot[mt % 1024] = slot[mt % 1024] + butterfly32(q);",
+     "slot[mt % 512] = slot[mt % 512] + butterfly32(q);"),
+    ("fitness tiles visited in decreasing order", "for (int64_t mt = 0; mt < tiles; ++mt) {",
+     "for (int64_t mt = tiles - 1; mt >= 0; --mt) {"),
+    ("fitness slots of a group added one after another", "double gsum = butterfly32(a);",
+     "double gsum = a[0]; for (int l = 1; l < 32; ++l) gsum = gsum + a[l];"),
+    ("fitness group sums added in reverse", _GROUPS_IN_ORDER,
+     _GROUPS_IN_ORDER.replace("int grp = 0; grp < 32; ++grp", "int grp = 31; grp >= 0; --grp")
+                     .replace("(grp == 0) ?", "(grp == 31) ?")),
+    ("fitness group sums combined by a butterfly", "total = (grp == 0) ? gsum : total + gsum;",
+     "slot[grp] = gsum; if (grp == 31) total = butterfly32(slot);"),
+    ("fitness term evaluated as (d*e)*e", "float e2 = e * e;\n    float term = dvec[j] * e2;",
+     "float term = (dvec[j] * e) * e;"),
+    ("fitness term evaluated in fp64", "return (double)term;",
+     "(void)term; { double ed = (double)x[j] - (double)tvec[j]; return (double)(float)((double)dvec[j] * (ed * ed)); }"),
+    ("fitness square kept in fp64", "float term = dvec[j] * e2;",
+     "(void)e2; float term = (float)((double)dvec[j] * ((double)e * (double)e));"),
 ]
 
 

@@ -433,6 +433,29 @@ def test_quadratic_fitness_special_cases():
     assert float(oracle.quadratic_fitness(xi, di, ti)) == float(np.sum(di * (xi - ti) ** 2))
 
 
+def _fitness_order_cases():
+    import golden_cases
+    return golden_cases.fitness_order_cases()
+
+
+@pytest.mark.parametrize("case", _fitness_order_cases(), ids=lambda c: c[0])
+def test_quadratic_fitness_hand_worked_order_and_rounding(case):
+    """The summation order and the three unfused fp32 operations of a term are
+    part of the fitness' definition; each golden case is worked by hand from
+    dyadic numbers so that another order or another rounding gives a different
+    fp32 value."""
+    name, w, d, t, want = case
+    got = oracle.quadratic_fitness(w, d, t)
+    assert got.view(np.uint32) == want.view(np.uint32), (name, float(got), float(want))
+    # the per-row entry point goes through the same function (row stride > N)
+    rows = np.zeros((3, w.size + 5), np.float32)
+    rows[1, :w.size] = w
+    rows[2, :w.size] = t                      # w = t: every error is 0
+    got_rows = oracle.quadratic_losses(rows[:, :w.size], d, t, nthreads=2)
+    assert got_rows[1].view(np.uint32) == want.view(np.uint32)
+    assert got_rows[2] == 0.0
+
+
 def test_quadratic_losses_rows():
     rng = np.random.default_rng(9)
     x = rng.standard_normal((5, 260)).astype(np.float32)
