@@ -9,6 +9,12 @@ the K losses, selection kernel, fused update kernel (psops_set_losses +
 psops_sync).  The metric is particle-elements updated per second; the roofline
 object relates the fused update kernel's algorithmic bytes to the measured HBM
 copy bandwidth of this machine's B200s.  Rank 0 prints one JSON line.
+
+The line certifies what it timed: after the timed region the state the GPU was
+left with is compared, on a seeded sample of columns, with the CPU oracle run
+from the same initial state through the same number of syncs ("parity"); a
+mismatch sets "parity_ok": false, is reported on stderr and makes the exit
+status non-zero.  The oracle never runs inside a timed region.
 """
 from __future__ import annotations
 
@@ -62,6 +68,12 @@ def parse_args():
     ap.add_argument("--row-steps", type=int, default=0,
                     help="timed steps per extra row (default 100, 50 for cfg5); with --n for small captures")
     ap.add_argument("--cpu-baseline", choices=["on", "off"], default="on")
+    ap.add_argument("--min-seconds", type=float, default=0.25,
+                    help="after the K timed steps, repeat K-step windows until this much device time has been "
+                         "measured in total (their spread is reported; the headline uses the first K steps)")
+    ap.add_argument("--parity", choices=["on", "off"], default="on",
+                    help="compare the timed state with the CPU oracle on a column sample")
+    ap.add_argument("--pieces", type=int, default=6, help="--parallelism shards: ranges of the gBest broadcast")
     ap.add_argument("--parallelism", choices=["replicas", "shards"], default="replicas",
                     help="shards: ONE swarm split by particle over the ranks (all-gather of losses + "
                          "broadcast of the best row per sync); strong scaling, not the default metric")
@@ -161,52 +173,109 @@ class ClockSampler:
 # ---------------------------------------------------------------------------
 # GPU arm
 # ---------------------------------------------------------------------------
-def device_state(w, dev):
-    """Upload the seeded recipe row by row: (x, v, pbest) as (K, ld) tensors."""
+def device_state(w, dev, cols=None):
+    """Upload the seeded recipe row by row: (x, v, pbest) as (K, ld) tensors.
+    With `cols` also returns the initial (x, v) at those columns as numpy
+    arrays, taken from the host rows before they are uploaded."""
     import torch
     from paper_2009_03816_b200 import workloads
     dx = torch.zeros((w.K, w.ld), dtype=torch.float32, device=dev)
     dv = torch.zeros((w.K, w.ld), dtype=torch.float32, device=dev)
+    xs = np.zeros((w.K, 0 if cols is None else cols.size), np.float32)
+    vs = np.zeros_like(xs)
     for k in range(w.K):
-        dx[k, :w.N] = torch.from_numpy(workloads.x_row(w, k)).to(dev)
+        row = workloads.x_row(w, k)
+        if cols is not None:
+            xs[k] = row[cols]
+        dx[k, :w.N] = torch.from_numpy(row).to(dev)
         if w.sigma_v != 0.0:
-            dv[k, :w.N] = torch.from_numpy(workloads.v_row(w, k)).to(dev)
-    return dx, dv, dx.clone()
+            row = workloads.v_row(w, k)
+            if cols is not None:
+                vs[k] = row[cols]
+            dv[k, :w.N] = torch.from_numpy(row).to(dev)
+    if cols is None:
+        return dx, dv, dx.clone()
+    return dx, dv, dx.clone(), xs, vs
 
 
-def make_swarm(w, dev, flags=0):
+def make_swarm(w, dev, flags=0, cols=None):
     from paper_2009_03816_b200 import binding
-    dx, dv, dp = device_state(w, dev)
+    dx, dv, dp, *sample = device_state(w, dev, cols)
     sw = binding.Swarm(dx, dv, dp, N=w.N, m_max=w.omega, m_min=w.omega, c1=w.c1, c2=w.c2,
                        seed=w.seed, flags=flags)
+    sw.initial_sample = tuple(sample) if sample else None
     return sw
 
 
-def time_region(fn, steps, warmup, ranks, sampler=None, counter=None):
+class Timing:
+    """Device times of one timed region (CUDA events on the current stream)."""
+
+    def __init__(self, seconds, step_ms=None):
+        self.seconds = seconds                # first event to last event: the K steps of the contract
+        self.step_ms = step_ms                # per-step durations, when every step had its own event pair
+        self.window_ms_per_step = []          # further K-step windows, if any
+
+    def stats(self, steps):
+        out = {"ms_per_step_mean": self.seconds * 1e3 / steps}
+        if self.step_ms:
+            a = np.asarray(self.step_ms)
+            out["per_step_ms"] = {"median": float(np.median(a)), "min": float(a.min()), "max": float(a.max()),
+                                  "n": int(a.size)}
+        if self.window_ms_per_step:
+            a = np.asarray([self.seconds * 1e3 / steps] + self.window_ms_per_step)
+            out["window_ms_per_step"] = {"median": float(np.median(a)), "min": float(a.min()),
+                                         "max": float(a.max()), "n": int(a.size)}
+        return out
+
+
+def time_region(fn, steps, warmup, ranks, sampler=None, counter=None, per_step=False, min_seconds=0.0,
+                first=0):
     """Warm up, then time exactly `steps` calls of fn(i) between barriers and
-    device synchronisation, with CUDA events on the current stream.  Returns
-    this rank's elapsed seconds (and, with `counter`, how much that counter
-    advanced inside the timed region)."""
+    device synchronisation, with CUDA events on the current stream (one pair
+    around the region; with per_step one event between any two steps as well).
+    If that measured less than min_seconds, further windows of `steps` calls
+    follow (each between its own event pair) until the total reaches it.
+    Returns (Timing, calls made, counter advance inside the first region)."""
     import torch
     from paper_2009_03816_b200 import replicas
-    for i in range(warmup):
+    i = first
+    for _ in range(warmup):
         fn(i)
+        i += 1
     torch.cuda.synchronize()
     replicas.barrier(ranks)
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1 if per_step else 2)]
     ctx = sampler if sampler is not None else _Null()
     c0 = counter() if counter is not None else 0
     with ctx:
-        e0.record()
-        for i in range(steps):
-            fn(warmup + i)
-        e1.record()
+        marks[0].record()
+        for k in range(steps):
+            fn(i)
+            i += 1
+            if per_step:
+                marks[k + 1].record()
+        if not per_step:
+            marks[1].record()
         torch.cuda.synchronize()
-    c1 = counter() if counter is not None else 0
-    replicas.barrier(ranks)
-    seconds = e0.elapsed_time(e1) * 1e-3
-    return (seconds, c1 - c0) if counter is not None else seconds
+        c1 = counter() if counter is not None else 0
+        replicas.barrier(ranks)
+        timing = Timing(marks[0].elapsed_time(marks[-1]) * 1e-3,
+                        [marks[k].elapsed_time(marks[k + 1]) for k in range(steps)] if per_step else None)
+        total = replicas.max_over_ranks(ranks, timing.seconds)
+        while total < min_seconds and len(timing.window_ms_per_step) < 64:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(steps):
+                fn(i)
+                i += 1
+            e1.record()
+            torch.cuda.synchronize()
+            sec = e0.elapsed_time(e1) * 1e-3
+            # every rank must make the same number of windows: agree on the slowest total
+            total = replicas.max_over_ranks(ranks, total + sec) if ranks.world > 1 else total + sec
+            timing.window_ms_per_step.append(sec * 1e3 / steps)
+    return timing, i - first, c1 - c0
 
 
 class _Null:
@@ -217,12 +286,20 @@ class _Null:
         return False
 
 
-def time_sync_workload(w, dev, steps, warmup, ranks, sampler=None, fused_fitness=False):
+PARITY_COLUMNS = 4096       # random columns of the sample (plus every residue mod 1024, block edges, head and tail)
+PARITY_TAIL = 8             # further syncs after the timed region whose selection is compared one by one
+
+
+def time_sync_workload(w, dev, steps, warmup, ranks, sampler=None, fused_fitness=False, per_step=False,
+                       min_seconds=0.0, cols=None, flags=0):
+    """Time psops_set_losses + psops_sync on a fresh swarm of recipe `w`.
+    Returns (swarm, Timing, syncs made since the initial state, launches in the
+    first timed region, tensors to keep alive, device loss table)."""
     import torch
     from paper_2009_03816_b200 import binding, workloads
-    flags = binding.PSOPS_QUADRATIC if fused_fitness else 0
-    sw = make_swarm(w, dev, flags)
-    keep = None
+    flags |= binding.PSOPS_QUADRATIC if fused_fitness else 0
+    sw = make_swarm(w, dev, flags, cols)
+    keep = dtable = None
     if fused_fitness:
         d, t = workloads.quadratic_vectors(w)
         keep = (torch.from_numpy(d).to(dev), torch.from_numpy(t).to(dev))
@@ -232,13 +309,112 @@ def time_sync_workload(w, dev, steps, warmup, ranks, sampler=None, fused_fitness
         def step(i):
             sw.sync(0, w.lam)
     else:
-        table = torch.from_numpy(workloads.losses(w)).to(dev)
+        dtable = torch.from_numpy(workloads.losses(w)).to(dev)
 
         def step(i):
-            sw.set_losses(table[i % table.shape[0]])
+            sw.set_losses(dtable[i % dtable.shape[0]])
             sw.sync(0, w.lam)
-    seconds, launches = time_region(step, steps, warmup, ranks, sampler, counter=lambda: sw.launches)
-    return sw, seconds, launches, keep
+    timing, made, launches = time_region(step, steps, warmup, ranks, sampler, counter=lambda: sw.launches,
+                                         per_step=per_step, min_seconds=min_seconds)
+    return sw, timing, made, launches, keep, dtable
+
+
+def _rel_err(got, want):
+    """(max relative error, elements outside 1e-6, elements not bit-identical)
+    under the parity contract |gpu - ref| <= 1e-6 max(|ref|, 1e-6 RMS(ref))."""
+    rms = float(np.sqrt(np.mean(np.square(want, dtype=np.float64)))) if want.size else 0.0
+    scale = np.maximum(np.abs(want).astype(np.float64), 1e-6 * rms if rms > 0 else 1e-300)
+    err = np.abs(got.astype(np.float64) - want.astype(np.float64)) / scale
+    same = (got.view(np.uint32) == want.view(np.uint32)) | ((got == 0) & (want == 0))
+    err = np.where(same, 0.0, err)
+    return float(np.nanmax(err)) if err.size else 0.0, int((~(err <= 1e-6)).sum()), int((~same).sum())
+
+
+def parity_after_timing(w, sw, made, cols, dtable, dev):
+    """Follow the sampled columns through the same `made` syncs in the CPU
+    oracle (outside any timed region) and compare with the state the GPU is
+    in; then PARITY_TAIL further syncs on both sides with the selection
+    compared after each."""
+    import torch
+    import oracle
+    from paper_2009_03816_b200 import workloads
+    xs, vs = sw.initial_sample
+    table = workloads.losses(w)
+    ref = oracle.RefSwarm(xs, vs, xs, m_max=w.omega, m_min=w.omega, t_max=1, c1=w.c1, c2=w.c2, seed=w.seed,
+                          elem_index=cols, nthreads=os.cpu_count() or 1)
+    for i in range(made):
+        ref.sync(table[i % table.shape[0]], 0, w.lam)
+    dcols = torch.from_numpy(cols).to(dev)
+
+    def selection_mismatch():
+        g, improved, pl = sw.info()
+        return int(g != ref.g or not np.array_equal(improved, ref.improved)
+                   or not np.array_equal(pl.view(np.uint32), ref.pbest_loss.view(np.uint32)))
+
+    def state():
+        worst, outside, inexact = 0.0, 0, 0
+        for t, want in ((sw.x, ref.x), (sw.v, ref.v), (sw.pbest, ref.p)):
+            e, o, n = _rel_err(t[:, dcols].cpu().numpy(), want)
+            worst, outside, inexact = max(worst, e), outside + o, inexact + n
+        return worst, outside, inexact
+
+    mism = selection_mismatch()
+    worst, outside, inexact = state()
+    for j in range(PARITY_TAIL):
+        i = made + j
+        sw.set_losses(dtable[i % dtable.shape[0]])
+        sw.sync(0, w.lam)
+        ref.sync(table[i % table.shape[0]], 0, w.lam)
+        mism += selection_mismatch()
+    e2, o2, n2 = state()
+    return {"ok": mism == 0 and outside + o2 == 0, "selection_mismatches": mism,
+            "max_rel_err": max(worst, e2), "outside_1e-6": outside + o2, "inexact": inexact + n2,
+            "columns": int(cols.size), "syncs": made + PARITY_TAIL,
+            "checked": f"x, v, pbest at the sampled columns after the {made} syncs made since the initial state "
+                       f"(warm-up, timed steps and windows) and again after {PARITY_TAIL} more; selection "
+                       f"(g, improved mask, pBest_loss) bit for bit after the last timed sync and after each of "
+                       f"the {PARITY_TAIL} (every earlier selection shaped the compared state)",
+            "oracle": "oracle/psops_ref.c, same initial state, same loss table"}
+
+
+def parity_fused_fitness(w, sw, keep, dev):
+    """cfg5-style rows: the losses come from the device, so the oracle needs the
+    whole swarm.  Take the state the timed region left, run ONE more sync on
+    both sides (oracle on all host cores) and compare the losses it consumed,
+    the selection, the new losses (bit for bit) and every element."""
+    import torch
+    import oracle
+    nthreads = os.cpu_count() or 1
+    N = w.N
+    x, v, p = (t[:, :N].cpu().numpy() for t in (sw.x, sw.v, sw.pbest))
+    d, t = (k.cpu().numpy() for k in keep)
+    _, pl = sw.state()
+    loss_gpu = sw.losses()
+    loss_ref = oracle.quadratic_losses(x, d, t, nthreads=nthreads)
+    mism = int(not np.array_equal(loss_gpu.view(np.uint32), loss_ref.view(np.uint32)))
+    step, _ = sw.state()
+    ref = oracle.RefSwarm(x, v, p, m_max=w.omega, m_min=w.omega, t_max=1, c1=w.c1, c2=w.c2, seed=w.seed,
+                          nthreads=nthreads)
+    ref.pbest_loss[:] = pl
+    ref.s = step
+    del x, v, p
+    sw.sync(0, w.lam)
+    ref.sync(loss_ref, 0, w.lam)
+    g, improved, pl2 = sw.info()
+    mism += int(g != ref.g or not np.array_equal(improved, ref.improved)
+                or not np.array_equal(pl2.view(np.uint32), ref.pbest_loss.view(np.uint32)))
+    new_ref = oracle.quadratic_losses(ref.x, d, t, nthreads=nthreads)
+    mism += int(not np.array_equal(sw.losses().view(np.uint32), new_ref.view(np.uint32)))
+    worst, outside, inexact = 0.0, 0, 0
+    for tdev, want in ((sw.x, ref.x), (sw.v, ref.v), (sw.pbest, ref.p)):
+        for k in range(w.K):                    # row by row keeps the host copies small
+            e, o, n = _rel_err(tdev[k, :N].cpu().numpy(), want[k])
+            worst, outside, inexact = max(worst, e), outside + o, inexact + n
+    return {"ok": mism == 0 and outside == 0, "selection_mismatches": mism, "max_rel_err": worst,
+            "outside_1e-6": outside, "inexact": inexact, "columns": int(N), "syncs": 1,
+            "checked": "one further sync from the state the timed region left, whole swarm in the oracle: the "
+                       "device-evaluated losses before and after it bit for bit, selection, every element of "
+                       "x, v, pbest"}
 
 
 def run_psops(args):
@@ -266,10 +442,18 @@ def run_psops(args):
         return
     sampler = ClockSampler(dev_index)
     fused = w.quadratic
-    sw, seconds, launches, keep = time_sync_workload(w, dev, args.steps, args.warmup, ranks, sampler, fused)
+    check = args.parity == "on" and ranks.is_root
+    cols = workloads.sample_columns_dense(w.N, PARITY_COLUMNS, w.seed) if check and not fused else None
+    sw, timing, made, launches, keep, dtable = time_sync_workload(
+        w, dev, args.steps, args.warmup, ranks, sampler, fused, per_step=pe >= 50_000_000,
+        min_seconds=args.min_seconds, cols=cols)
+    seconds = timing.seconds
     rate, slowest = replicas.whole_job_rate(ranks, pe * args.steps, seconds)
     ms_per_step = slowest * 1e3 / args.steps
     achieved = sync_bytes(w, fused) / (seconds / args.steps) / 1e9
+    parity = None
+    if check:
+        parity = parity_fused_fitness(w, sw, keep, dev) if fused else parity_after_timing(w, sw, made, cols, dtable, dev)
 
     # ---- end to end: host buffers in, host buffers out, through psops_sync_host
     e2e = None
@@ -306,8 +490,10 @@ def run_psops(args):
         "config": {"workload": f"{w.name}: K={w.K} particles x N={w.N} fp32 ({w.note}), "
                                f"omega={w.omega}, c1={w.c1}, c2={w.c2}, lambda={w.lam}, seed={w.seed}",
                    "K": w.K, "N": w.N, "ld": w.ld, "replicas": ranks.world,
-                   "l2": "state (12*K*N bytes) exceeds L2; no flush needed",
+                   "l2": "state (12*K*N bytes) exceeds L2; no flush needed" if 12 * pe > (126 << 20)
+                         else "state fits L2: an L2-resident result, reported as such",
                    "parallelism": "replicas only"},
+        "timing": timing.stats(args.steps),
         "clocks": sampler.report(),
         "e2e": e2e,
         "gpu_launches": int(replicas.sum_over_ranks(ranks, launches)),
@@ -315,7 +501,11 @@ def run_psops(args):
                      "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal_8TBs": achieved / 8000.0,
                      "bytes_per_launch": sync_bytes(w, fused), "traffic": ncu_traffic(w),
-                     "note": "duration = timed region / steps (includes the selection kernel)"},
+                     "note": "duration = timed region / steps (includes the selection kernel); the peak is a "
+                             "measured 1:1 copy, which this 3:2 read:write kernel can exceed slightly -- "
+                             "frac_of_nominal_8TBs is the fraction of the nominal HBM3e rate"},
+        "parity": parity,
+        "parity_ok": None if parity is None else bool(parity["ok"]),
     }
     sw.close()
     del sw, keep
@@ -324,16 +514,27 @@ def run_psops(args):
     if ranks.is_root and ranks.world == 1:
         if args.rows == "all":
             out["rows"] = other_rows(args, dev, ranks, peak)
+            bad = [k for k, r in out["rows"].items() if isinstance(r, dict) and r.get("parity") and not r["parity"]["ok"]]
+            if bad:
+                out["parity_ok"] = False
+                out["parity_failed_rows"] = bad
         if args.cpu_baseline == "on":
             out["cpu_baseline"] = cpu_baseline(w)
     if ranks.is_root:
         print(json.dumps(out), flush=True)
+        if out["parity_ok"] is False:
+            print("PARITY FAILURE: the timed state does not match the oracle: "
+                  + json.dumps({"headline": parity, "rows": out.get("parity_failed_rows")}), file=sys.stderr, flush=True)
     replicas.finish(ranks)
+    if out["parity_ok"] is False:
+        raise SystemExit(3)
 
 
 def run_shards(args, w, dev, dev_index, ranks, peak, peak_src):
     """One swarm, K / world particles per rank.  Per sync every rank receives
-    4 K bytes of losses and 4 N bytes of gBest instead of the other ranks' rows."""
+    4 K bytes of losses and 4 N bytes of gBest instead of the other ranks' rows;
+    the broadcast travels in --pieces element ranges and the update of a range
+    runs while the next one is on the wire."""
     import torch
     from paper_2009_03816_b200 import binding, replicas, sharded, workloads
     if w.K % ranks.world or w.quadratic:
@@ -349,17 +550,24 @@ def run_shards(args, w, dev, dev_index, ranks, peak, peak_src):
             dv[r, :w.N] = torch.from_numpy(workloads.v_row(w, first + r)).to(dev)
     sw = binding.Swarm(dx, dv, dx.clone(), N=w.N, m_max=w.omega, m_min=w.omega, c1=w.c1, c2=w.c2,
                        seed=w.seed, k_first=first, K_total=w.K)
-    drv = sharded.ShardedSync(sharded.swarm_engine(sw), counts, w.N, dev)
+    drv = sharded.ShardedSync(sharded.swarm_engine(sw), counts, w.N, dev, pieces=args.pieces, timing=True)
     table = torch.from_numpy(workloads.losses(w)).to(dev)
     sampler = ClockSampler(dev_index)
 
     def step(i):
         drv.sync(table[i % table.shape[0], first:first + n_here], 0, w.lam)
 
-    seconds, launches = time_region(step, args.steps, args.warmup, ranks, sampler, counter=lambda: sw.launches)
+    for i in range(args.warmup):
+        step(i)
+    drv.timings_ms()                                 # drop the warm-up's events
+    timing, _, launches = time_region(step, args.steps, 0, ranks, sampler, counter=lambda: sw.launches,
+                                      first=args.warmup)
+    phases = drv.timings_ms()
+    seconds = timing.seconds
     slowest = replicas.max_over_ranks(ranks, seconds)
     bytes_here = 20 * n_here * w.N + 4 * w.N
     achieved = bytes_here / (seconds / args.steps) / 1e9
+    phases = {k: (replicas.max_over_ranks(ranks, v) if isinstance(v, float) else v) for k, v in phases.items()}
     out = {
         "metric": METRIC, "value": w.K * w.N * args.steps / slowest, "unit": UNIT, "n_gpus": ranks.world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": slowest * 1e3 / args.steps,
@@ -367,14 +575,15 @@ def run_shards(args, w, dev, dev_index, ranks, peak, peak_src):
         "data": "synthetic",
         "config": {"workload": f"{w.name}: K={w.K} particles x N={w.N} fp32 ({w.note}), one swarm sharded by particle",
                    "K": w.K, "N": w.N, "ld": w.ld, "particles_per_rank": n_here,
-                   "parallelism": f"particle shards x{ranks.world}",
+                   "parallelism": f"particle shards x{ranks.world}", "broadcast_pieces": len(drv.bounds),
                    "exchange_bytes_per_rank_per_sync": sharded.bytes_received_per_sync(w.N, counts)},
+        "phases_ms_per_sync_max_over_ranks": phases,
         "clocks": sampler.report(), "e2e": None,
         "gpu_launches": int(replicas.sum_over_ranks(ranks, launches)),
         "roofline": {"bound": "hbm", "kernel": "psops_update_kernel", "achieved": achieved, "peak": peak,
                      "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
                      "bytes_per_launch": bytes_here, "traffic": None,
-                     "note": "duration = timed region / steps: collectives, selection (with its host read of g) "
+                     "note": "duration = timed region / steps: collectives, selection (with the host's read of g) "
                              "and update of this rank's particles"},
     }
     sw.close()
@@ -427,6 +636,16 @@ def graph_us_per_sync(w, dev, replays=20):
     return e0.elapsed_time(e1) * 1e3 / (replays * len(rows))
 
 
+def _row(w, timing, steps, nbytes, peak, K_here=None, parity=None):
+    sec = timing.seconds
+    gbs = nbytes / (sec / steps) / 1e9
+    out = {"ms_per_step": sec * 1e3 / steps, "value": (K_here or w.K) * w.N * steps / sec, "unit": UNIT,
+           "GBps": gbs, "frac": gbs / peak, "frac_of_nominal_8TBs": gbs / 8000.0, "timing": timing.stats(steps)}
+    if parity is not None:
+        out["parity"] = parity
+    return out
+
+
 def time_variant(w, dev, ranks, peak, flags=0, shard=None, steps=100):
     """psops_sync with a flag set, or the select + update pair of one particle shard."""
     import torch
@@ -450,13 +669,12 @@ def time_variant(w, dev, ranks, peak, flags=0, shard=None, steps=100):
             sw.set_losses(table[i % table.shape[0]])
             sw.shard_select()
             sw.shard_update(gbest, 0, w.lam)
-    sec = time_region(step, steps, 5, ranks)
-    gbs = (20 * K_here * w.N + 4 * w.N) / (sec / steps) / 1e9
+    timing, _, _ = time_region(step, steps, 5, ranks, per_step=True, min_seconds=0.05)
+    out = _row(w, timing, steps, 20 * K_here * w.N + 4 * w.N, peak, K_here)
     sw.close()
     del sw
     torch.cuda.empty_cache()
-    return {"ms_per_step": sec * 1e3 / steps, "value": K_here * w.N * steps / sec, "unit": UNIT,
-            "GBps": gbs, "frac": gbs / peak}
+    return out
 
 
 def other_rows(args, dev, ranks, peak):
@@ -464,25 +682,25 @@ def other_rows(args, dev, ranks, peak):
     import torch
     from paper_2009_03816_b200 import workloads
     rows = {}
+    check = args.parity == "on"
     try:
         w3, w5 = workloads.CONFIGS["cfg3"], workloads.CONFIGS["cfg5"]
         if args.n:
             w3, w5 = w3.scaled(N=args.n), w5.scaled(N=args.n)
         S3, S5, W = args.row_steps or 100, args.row_steps or 50, (5 if not args.row_steps else 3)
-        sw, sec, _, _ = time_sync_workload(w3, dev, S3, W, ranks)
-        gbs = sync_bytes(w3) / (sec / S3) / 1e9
-        rows["cfg3_sync"] = {"ms_per_step": sec * 1e3 / S3, "value": w3.K * w3.N * S3 / sec, "unit": UNIT,
-                             "GBps": gbs, "frac": gbs / peak}
-        sec = time_region(lambda i: sw.average(), S3, W, ranks)
-        gbs = average_bytes(w3) / (sec / S3) / 1e9
-        rows["cfg3_average"] = {"ms_per_step": sec * 1e3 / S3, "value": w3.K * w3.N * S3 / sec, "unit": UNIT,
-                                "GBps": gbs, "frac": gbs / peak}
+        cols = workloads.sample_columns_dense(w3.N, PARITY_COLUMNS, w3.seed) if check else None
+        sw, timing, made, _, _, dtable = time_sync_workload(w3, dev, S3, W, ranks, per_step=True,
+                                                            min_seconds=0.1, cols=cols)
+        par = parity_after_timing(w3, sw, made, cols, dtable, dev) if check else None
+        rows["cfg3_sync"] = _row(w3, timing, S3, sync_bytes(w3), peak, parity=par)
+        timing, _, _ = time_region(lambda i: sw.average(), S3, W, ranks, per_step=True)
+        rows["cfg3_average"] = _row(w3, timing, S3, average_bytes(w3), peak)
+        if check:       # every row of x must now hold the same values: spot-check against row 0
+            rows["cfg3_average"]["rows_equal"] = bool(torch.equal(sw.x[0, :w3.N], sw.x[w3.K - 1, :w3.N]))
         # SSGD baseline on the same rows: K gradient rows in, K weight rows out
         grad = torch.randn((w3.K, w3.ld), device=dev, generator=torch.Generator(device=dev).manual_seed(3))
-        sec = time_region(lambda i: sw.ssgd(grad, -0.01), S3, W, ranks)
-        gbs = (8 * w3.K * w3.N + 4 * w3.N) / (sec / S3) / 1e9
-        rows["cfg3_ssgd"] = {"ms_per_step": sec * 1e3 / S3, "value": w3.K * w3.N * S3 / sec, "unit": UNIT,
-                             "GBps": gbs, "frac": gbs / peak}
+        timing, _, _ = time_region(lambda i: sw.ssgd(grad, -0.01), S3, W, ranks, per_step=True)
+        rows["cfg3_ssgd"] = _row(w3, timing, S3, 8 * w3.K * w3.N + 4 * w3.N, peak)
         del grad
         sw.close()
         del sw
@@ -491,28 +709,33 @@ def other_rows(args, dev, ranks, peak):
         # what one GPU of an 8-GPU particle-sharded run does per sync: 2 of the 16 particles,
         # gBest read from a broadcast buffer (the collectives themselves need more than one GPU)
         rows["cfg3_shard_2_of_16"] = time_variant(w3, dev, ranks, peak, shard=(0, 2), steps=S3)
-        sw, sec, _, keep = time_sync_workload(w5, dev, S5, W, ranks, fused_fitness=True)
-        gbs = sync_bytes(w5, True) / (sec / S5) / 1e9
-        rows["cfg5_sync_fused_fitness"] = {"ms_per_step": sec * 1e3 / S5, "value": w5.K * w5.N * S5 / sec,
-                                           "unit": UNIT, "GBps": gbs, "frac": gbs / peak}
-        sec = time_region(lambda i: sw.eval_quadratic(), S5, W, ranks)
+        sw, timing, _, _, keep, _ = time_sync_workload(w5, dev, S5, W, ranks, fused_fitness=True, per_step=True)
+        par = parity_fused_fitness(w5, sw, keep, dev) if check else None
+        rows["cfg5_sync_fused_fitness"] = _row(w5, timing, S5, sync_bytes(w5, True), peak, parity=par)
+        timing, _, _ = time_region(lambda i: sw.eval_quadratic(), S5, W, ranks, per_step=True)
         tiles = (w5.N + 127) // 128
-        gbs = (4 * w5.K * w5.N + 8 * w5.N + 16 * w5.K * tiles) / (sec / S5) / 1e9
-        rows["cfg5_fitness_only"] = {"ms_per_step": sec * 1e3 / S5, "value": w5.K * w5.N * S5 / sec,
-                                     "unit": UNIT, "GBps": gbs, "frac": gbs / peak}
+        rows["cfg5_fitness_only"] = _row(w5, timing, S5, 4 * w5.K * w5.N + 8 * w5.N + 16 * w5.K * tiles, peak)
         sw.close()
         del sw, keep
         torch.cuda.empty_cache()
         for name in (() if args.n else ("cfg1", "cfg2")):
             ws = workloads.CONFIGS[name]
-            sw, sec, _, _ = time_sync_workload(ws, dev, 200, 10, ranks)
-            rows[name + "_sync"] = {"us_per_step": sec / 200 * 1e6, "value": ws.K * ws.N * 200 / sec,
-                                    "unit": UNIT, "note": "small case: host launch rate / L2-resident",
+            cols = workloads.sample_columns_dense(ws.N, PARITY_COLUMNS, ws.seed) if check else None
+            sw, timing, made, launches, _, dtable = time_sync_workload(ws, dev, 200, 10, ranks, min_seconds=0.05,
+                                                                       cols=cols)
+            st = timing.stats(200)
+            rows[name + "_sync"] = {"us_per_step": timing.seconds / 200 * 1e6, "value": ws.K * ws.N * 200 / timing.seconds,
+                                    "unit": UNIT, "launches_per_sync": launches / 200,
+                                    "GBps": sync_bytes(ws) / (timing.seconds / 200) / 1e9,
+                                    "note": "small case: host launch rate / L2-resident", "timing": st,
                                     "us_per_step_cuda_graph": graph_us_per_sync(ws, dev)}
+            if check:
+                rows[name + "_sync"]["parity"] = parity_after_timing(ws, sw, made, cols, dtable, dev)
             sw.close()
             del sw
     except Exception as exc:  # report, do not lose the headline line
-        rows["error"] = repr(exc)
+        import traceback
+        rows["error"] = repr(exc) + " | " + traceback.format_exc().splitlines()[-3].strip()
     return rows
 
 
@@ -544,11 +767,8 @@ def oracle_step(ref, w, table, d, t, i, nthreads):
     ref.sync(loss, 0, w.lam)
 
 
-def cpu_baseline(w, target_seconds=1.5, syncs=3):
-    """Time the oracle as it stands on this box's host cores on a bounded
-    sample of the workload's columns."""
-    nthreads = os.cpu_count() or 1
-    n_cols = 1 << 16
+def _time_oracle(w, nthreads, target_seconds, syncs):
+    n_cols = 1 << 14
     ref, table, d, t = oracle_sample(w, n_cols, nthreads)
     t0 = time.perf_counter()
     oracle_step(ref, w, table, d, t, 0, nthreads)
@@ -559,9 +779,21 @@ def cpu_baseline(w, target_seconds=1.5, syncs=3):
     for i in range(syncs):
         oracle_step(ref, w, table, d, t, i, nthreads)
     sec = time.perf_counter() - t0
-    return {"value": w.K * n_cols * syncs / sec, "unit": UNIT, "cores": nthreads, "kind": "oracle",
+    return w.K * n_cols * syncs / sec, n_cols, sec
+
+
+def cpu_baseline(w, target_seconds=1.5, syncs=3):
+    """Time the oracle as it stands on this box's host cores on a bounded
+    sample of the workload's columns: all cores (OpenMP over elements) and one
+    thread."""
+    nthreads = os.cpu_count() or 1
+    value, n_cols, sec = _time_oracle(w, nthreads, target_seconds, syncs)
+    value1, n_cols1, sec1 = _time_oracle(w, 1, target_seconds, syncs)
+    return {"value": value, "unit": UNIT, "cores": nthreads, "kind": "oracle",
             "sample": f"{syncs} syncs of the first {n_cols} of {w.N} columns, all K={w.K} particles, "
-                      f"OpenMP over elements", "seconds": sec}
+                      f"OpenMP over elements", "seconds": sec,
+            "one_thread": {"value": value1, "cores": 1, "seconds": sec1,
+                           "sample": f"{syncs} syncs of the first {n_cols1} of {w.N} columns"}}
 
 
 def run_reference(args):

@@ -61,6 +61,7 @@ extern "C" {
 #define PSOPS_KEEP_GBEST   1u  /* keep a copy of the gBest row of each sync (+4N bytes of workspace) */
 #define PSOPS_QUADRATIC    2u  /* reserve workspace for the on-device quadratic fitness              */
 #define PSOPS_GBEST_HISTORY 4u /* gBest = best of all syncs so far instead of this sync's best (+4N bytes) */
+#define PSOPS_SEPARATE_SELECT 8u /* always run the selection as a kernel of its own (see psops_sync)       */
 
 /* `which` of psops_get_weights / psops_set_weights */
 #define PSOPS_X      0         /* weights  w_i  (position of particle i)     */
@@ -80,7 +81,8 @@ typedef struct {
     int64_t  t_max;          /* Eq. 5 denominator (Max_t of Algorithm 1), >= 1              */
     float    c1, c2;         /* acceleration constants of Eq. 6                             */
     uint64_t seed;           /* Philox key                                                  */
-    uint32_t flags;          /* PSOPS_KEEP_GBEST | PSOPS_QUADRATIC | PSOPS_GBEST_HISTORY    */
+    uint32_t flags;          /* PSOPS_KEEP_GBEST | PSOPS_QUADRATIC | PSOPS_GBEST_HISTORY |
+                                PSOPS_SEPARATE_SELECT                                       */
     int32_t  K_total;        /* particles in the whole swarm when this context holds a shard
                                 [k_first, k_first + K) of it; 0 = not sharded (K_total = K)  */
 } psops_config;
@@ -134,6 +136,18 @@ int psops_set_losses(psops_ctx *ctx, const float *losses, int on_device);
  * psops_sync recorded into a CUDA graph (with the losses in a device buffer,
  * see psops_set_losses) keeps walking the random stream when the graph is
  * replayed; t_iter and lambda are then the ones given at capture.
+ * Launches: a small swarm -- at most 32 particles, no history variant, no fused
+ * fitness, and few enough elements that all thread blocks of the update are
+ * resident at once (about 450,000 on a B200) -- is launch-bound, and its whole
+ * sync is ONE kernel: every thread block recomputes steps 1 and 2 from the K
+ * losses, and the block that finishes last publishes g, the improved mask,
+ * pBest_loss and the counter (no block waits for another).  Otherwise, or with
+ * PSOPS_SEPARATE_SELECT, a selection kernel runs first and the update kernel
+ * behind it.  The results are identical bit for bit.
+ * Cache policy: a swarm whose state (12 bytes per particle-element) is at most
+ * three quarters of the GPU's L2 cache is accessed with ordinary loads and
+ * stores so that the next sync finds it there; larger swarms are streamed
+ * (evict-first).
  * Errors: EINVAL (t_iter < 0, lambda < 1 or not finite), ESTATE (no losses
  * yet), ECUDA.
  */
@@ -147,7 +161,10 @@ int psops_sync(psops_ctx *ctx, int64_t t_iter, float lambda);
  * the new weights (may equal h_x_in).  Velocities and personal bests stay on
  * the device.  Copies and kernels are pipelined over element ranges; the call
  * returns when h_x_out is complete.  Pinned host memory gives full speed.
- * Errors: as psops_sync, plus ENAN.
+ * Errors: as psops_sync, plus ENAN.  Also on an error from the CUDA runtime the
+ * call returns only after every copy and kernel it had queued has finished, so
+ * the host buffers may be freed at once; the swarm's state is then undefined
+ * (some element ranges updated, others not).
  */
 int psops_sync_host(psops_ctx *ctx, const float *h_x_in, int64_t h_in_ld,
                     const float *h_losses, int64_t t_iter, float lambda,
@@ -177,13 +194,29 @@ int psops_host_unregister(void *host_ptr);
  *   4. psops_shard_update: Eq. 6 / Eq. 7 for this shard's particles with gBest
  *      read from d_gbest_row (N floats, device pointer, 16-byte aligned on the
  *      128-bit path).  Random draws use the swarm-wide particle index, so the
- *      result is that of one unsharded psops_sync.
- * psops_sync itself returns ESTATE on a sharded context.  The quadratic
- * fitness and PSOPS_GBEST_HISTORY are not available on shards.
- * Errors: EINVAL, EALIGN, ESTATE (no losses / update without select), ECUDA.
+ *      result is that of one unsharded psops_sync.  The shard that holds
+ *      particle g may pass that row of its own x directly: every element of
+ *      gBest is read by the thread that later overwrites it.
+ *      psops_shard_update_range does step 4 for elements [first_elem,
+ *      last_elem) only, so that the broadcast can travel in pieces and the
+ *      update of one piece runs while the next is still on the wire: call it
+ *      with consecutive ranges from 0 to N (first_elem a multiple of 4,
+ *      last_elem a multiple of 4 or N; d_gbest_row always points at element 0 of
+ *      the row, of which only the range is read); the sync counter advances when
+ *      the range that ends at N has been enqueued.
+ * psops_shard_select waits only for the selection kernel (an event behind it;
+ * g arrives through a page-locked word the kernel writes), not for later work.
+ * psops_sync, psops_sync_host, psops_average and psops_ssgd return ESTATE on a
+ * sharded context (they need the whole swarm).  The quadratic fitness and
+ * PSOPS_GBEST_HISTORY are not available on shards; PSOPS_KEEP_GBEST is (the
+ * shard keeps a copy of the row it was given).
+ * Errors: EINVAL, EALIGN, ESTATE (no losses / update without select / a range
+ * out of order), ECUDA.
  */
 int psops_shard_select(psops_ctx *ctx, int *g);
 int psops_shard_update(psops_ctx *ctx, int64_t t_iter, float lambda, const float *d_gbest_row);
+int psops_shard_update_range(psops_ctx *ctx, int64_t t_iter, float lambda, const float *d_gbest_row,
+                             int64_t first_elem, int64_t last_elem);
 
 /*
  * gBest from the history of all particles (the standard-PSO framework of
@@ -273,8 +306,13 @@ int psops_eval_quadratic(psops_ctx *ctx);
  * much memory on every GPU that loads it until the process exits.  A problem
  * with K * ceil(N/128) above that number is refused with PSOPS_ELIMIT and
  * nothing is launched.  The first call on each device looks the array's address
- * up (the device must be current) -- make that first call outside any stream
- * capture.  All calls on a device share the array and it is not cleared
+ * up (the device on which the pointers live must be current, then and in every
+ * later call) -- make that first call outside any stream capture and at
+ * start-up: if nothing else of this library has run on the device yet, it is
+ * also the moment the CUDA runtime loads the library's device code and reserves
+ * the 8 MiB, which may synchronise the device and, on a GPU with no memory
+ * left, fail.  Such a failure is returned as PSOPS_ECUDA (there is no context
+ * to hold a message; cudaGetLastError has been cleared).  All calls on a device share the array and it is not cleared
  * between calls (every slot that is read has been written by the same call);
  * calls that overlap in time on one GPU overwrite each other's partial results,
  * so keep them on one stream or order them yourself.

@@ -21,7 +21,7 @@ PSOPS_EINVAL, PSOPS_EALIGN, PSOPS_ESTATE, PSOPS_ENAN = -1, -2, -3, -4
 PSOPS_EWORKSPACE, PSOPS_ECUDA, PSOPS_ENOMEM, PSOPS_ELIMIT = -5, -6, -7, -8
 PSOPS_STATIC_SCRATCH_DOUBLES = 1 << 20
 PSOPS_MAX_K = 1024
-PSOPS_KEEP_GBEST, PSOPS_QUADRATIC, PSOPS_GBEST_HISTORY = 1, 2, 4
+PSOPS_KEEP_GBEST, PSOPS_QUADRATIC, PSOPS_GBEST_HISTORY, PSOPS_SEPARATE_SELECT = 1, 2, 4, 8
 PSOPS_X, PSOPS_V, PSOPS_PBEST, PSOPS_GBEST = 0, 1, 2, 3
 
 EXPORTS = [
@@ -31,7 +31,7 @@ EXPORTS = [
     "psops_eval_quadratic", "psops_get_state", "psops_set_state", "psops_inertia",
     "psops_launch_count", "psops_strerror", "psops_last_error", "psops_destroy",
     "psops_quadratic_fitness_static", "psops_shard_select", "psops_shard_update",
-    "psops_get_history", "psops_set_history", "psops_ssgd",
+    "psops_shard_update_range", "psops_get_history", "psops_set_history", "psops_ssgd",
     "psops_host_register", "psops_host_unregister",
 ]
 
@@ -92,6 +92,8 @@ def load() -> ctypes.CDLL:
         "psops_destroy": (ctypes.c_int, [_vp]),
         "psops_shard_select": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_int)]),
         "psops_shard_update": (ctypes.c_int, [_vp, ctypes.c_int64, ctypes.c_float, _f32p]),
+        "psops_shard_update_range": (ctypes.c_int, [_vp, ctypes.c_int64, ctypes.c_float, _f32p,
+                                                    ctypes.c_int64, ctypes.c_int64]),
         "psops_get_history": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int)]),
         "psops_set_history": (ctypes.c_int, [_vp, ctypes.c_float, _f32p, ctypes.c_int]),
         "psops_ssgd": (ctypes.c_int, [_vp, _f32p, ctypes.c_int64, ctypes.c_float]),
@@ -189,6 +191,12 @@ def psops_shard_select(ctx) -> int:
 def psops_shard_update(ctx, t_iter, lam, d_gbest_row) -> None:
     _check(load().psops_shard_update(ctx, int(t_iter), float(lam), _ptr(d_gbest_row)),
            "psops_shard_update", ctx)
+
+
+def psops_shard_update_range(ctx, t_iter, lam, d_gbest_row, first_elem, last_elem) -> None:
+    _check(load().psops_shard_update_range(ctx, int(t_iter), float(lam), _ptr(d_gbest_row),
+                                           int(first_elem), int(last_elem)),
+           "psops_shard_update_range", ctx)
 
 
 def psops_get_history(ctx):
@@ -337,6 +345,9 @@ class Swarm:
 
     def shard_update(self, d_gbest_row, t_iter=0, lam=1.0):
         psops_shard_update(self.ctx, t_iter, lam, d_gbest_row)
+
+    def shard_update_range(self, d_gbest_row, first_elem, last_elem, t_iter=0, lam=1.0):
+        psops_shard_update_range(self.ctx, t_iter, lam, d_gbest_row, first_elem, last_elem)
 
     def ssgd(self, d_grad, alpha):
         psops_ssgd(self.ctx, d_grad, d_grad.stride(0), alpha)

@@ -27,6 +27,7 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "psops_kernels.cuh"
@@ -36,6 +37,13 @@
 // filling and draining the three-stage pipeline stays a small share.
 #ifndef PSOPS_HOST_CHUNK_BYTES
 #define PSOPS_HOST_CHUNK_BYTES (64ll << 20)
+#endif
+
+// A swarm whose state (12 bytes per particle-element) is at most this share of
+// the L2 cache is accessed with ordinary write-back loads and stores instead
+// of evict-first ones.
+#ifndef PSOPS_L2_RESIDENT_PERCENT
+#define PSOPS_L2_RESIDENT_PERCENT 75
 #endif
 
 namespace {
@@ -59,7 +67,7 @@ bool config_ok(const psops_config *c)
     if (c->t_max < 1) return false;
     if (!std::isfinite(c->m_max) || !std::isfinite(c->m_min)) return false;
     if (!std::isfinite(c->c1) || !std::isfinite(c->c2)) return false;
-    if (c->flags & ~(PSOPS_KEEP_GBEST | PSOPS_QUADRATIC | PSOPS_GBEST_HISTORY)) return false;
+    if (c->flags & ~(PSOPS_KEEP_GBEST | PSOPS_QUADRATIC | PSOPS_GBEST_HISTORY | PSOPS_SEPARATE_SELECT)) return false;
     // particle shard: rows [k_first, k_first + K) of a swarm of K_total particles
     if (c->K_total == 0) {
         if (c->k_first != 0) return false;
@@ -121,7 +129,13 @@ struct psops_ctx {
     bool aligned;
     bool have_losses;
     bool synced_once;
-    bool selected;                     // psops_shard_select ran and psops_shard_update has not yet
+    bool selected;                     // psops_shard_select ran and the update of that sync is not complete yet
+    long long range_next;              // first element the next psops_shard_update_range must start at
+    int *h_g;                          // page-locked, device-mapped word the selection kernel writes g to (shards)
+    int *d_g;                          // the same word as the device sees it
+    cudaEvent_t ev_select;             // recorded behind the selection kernel of a shard
+    bool stream_policy;                // true: evict-first accesses (state larger than L2)
+    long long one_wave_blocks;         // blocks of the select-in-update kernel that are resident at once on this GPU
     int Kt;                            // particles in the whole swarm (= cfg.K unless sharded)
     uint32_t step;                     // syncs enqueued through this context (the stream's own counter is on the device)
     long long quads, tiles;
@@ -185,12 +199,12 @@ void fill_round_keys(uint64_t seed, uint32_t (&rk)[20])
     }
 }
 
-int launch_select(psops_ctx *ctx)
+int launch_select(psops_ctx *ctx, int *g_mapped = nullptr)
 {
     const int threads = (int)round_up((size_t)ctx->Kt, 32);
     psops_select_kernel<<<1, threads, 0, ctx->stream>>>(ctx->loss_src, ctx->d_losses, ctx->d_pbest_loss,
                                                         ctx->d_desc, ctx->Kt,
-                                                        (ctx->cfg.flags & PSOPS_GBEST_HISTORY) ? 1 : 0);
+                                                        (ctx->cfg.flags & PSOPS_GBEST_HISTORY) ? 1 : 0, g_mapped);
     ctx->loss_src = ctx->d_losses;     // the kernel keeps a copy there
     return check_launch(ctx, "psops_select_kernel");
 }
@@ -200,26 +214,58 @@ constexpr int kFitUnroll = PSOPS_FITNESS_UNROLL, kFitQuads = PSOPS_FITNESS_QUADS
 static_assert(32 % kUnroll == 0 && 32 % kFitUnroll == 0, "the improved mask is reloaded every 32 particles");
 static_assert(kUpdateThreads % 32 == 0, "a warp must cover whole 128-element tiles");
 
-template <typename Kernel>
-cudaError_t launch_update_kernel(Kernel kernel, unsigned blocks, cudaStream_t stream, bool after_select,
-                                 const UpdateParams &P)
+// Launch with programmatic stream serialisation: the grid may become resident
+// while the kernel in front of it in the stream is still running; the kernel
+// itself waits (griddepcontrol.wait) for that kernel to finish before it reads
+// anything.  For a kernel that does not trigger early this is an ordinary launch.
+template <typename... Params, typename... Args>
+cudaError_t launch_serialized(bool programmatic, void (*kernel)(Params...), dim3 grid, dim3 block,
+                              cudaStream_t stream, Args &&...args)
 {
     cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(blocks, 1, 1);
-    cfg.blockDim = dim3(kUpdateThreads, 1, 1);
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
     cfg.dynamicSmemBytes = 0;
     cfg.stream = stream;
     cudaLaunchAttribute attr{};
     attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
-    cfg.numAttrs = after_select ? 1 : 0;   // overlap the launch with the selection kernel in front of it
-    return cudaLaunchKernelEx(&cfg, kernel, P);
+    cfg.numAttrs = programmatic ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
+using UpdateKernel = void (*)(const UpdateParams);
+
+// aligned | fitness << 1 | select << 2 | stream << 3  (select and fitness never together)
+UpdateKernel pick_update_kernel(bool aligned, bool fitness, bool select, bool stream)
+{
+    static const UpdateKernel table[16] = {
+        psops_update_kernel<false, false, false, false, kUnroll, kQuads>,
+        psops_update_kernel<true, false, false, false, kUnroll, kQuads>,
+        psops_update_kernel<false, true, false, false, kFitUnroll, kFitQuads>,
+        psops_update_kernel<true, true, false, false, kFitUnroll, kFitQuads>,
+        psops_update_kernel<false, false, true, false, kUnroll, kQuads>,
+        psops_update_kernel<true, false, true, false, kUnroll, kQuads>,
+        nullptr,
+        nullptr,
+        psops_update_kernel<false, false, false, true, kUnroll, kQuads>,
+        psops_update_kernel<true, false, false, true, kUnroll, kQuads>,
+        psops_update_kernel<false, true, false, true, kFitUnroll, kFitQuads>,
+        psops_update_kernel<true, true, false, true, kFitUnroll, kFitQuads>,
+        psops_update_kernel<false, false, true, true, kUnroll, kQuads>,
+        psops_update_kernel<true, false, true, true, kUnroll, kQuads>,
+        nullptr,
+        nullptr,
+    };
+    return table[(aligned ? 1 : 0) | (fitness ? 2 : 0) | (select ? 4 : 0) | (stream ? 8 : 0)];
+}
+
+// One launch of kernel (b) over quads [q_begin, q_end).  `select`: the launch
+// also does the selection of this sync (whole range, K <= 32, see the kernel).
 int launch_update(psops_ctx *ctx, float m, float k1, float k2, long long q_begin,
-                  long long q_end, bool fitness, cudaStream_t stream, bool after_select = false,
-                  const float *gbest_ext = nullptr)
+                  long long q_end, bool fitness, cudaStream_t stream, bool programmatic = false,
+                  bool select = false, const float *gbest_ext = nullptr)
 {
     if (q_end <= q_begin) return PSOPS_OK;
     UpdateParams P{};
@@ -229,6 +275,8 @@ int launch_update(psops_ctx *ctx, float m, float k1, float k2, long long q_begin
     P.i_first = ctx->cfg.k_first;
     P.dvec = ctx->dvec; P.tvec = ctx->tvec; P.partials = ctx->d_partials;
     P.desc = ctx->d_desc;
+    P.loss_src = ctx->loss_src; P.loss_keep = ctx->d_losses; P.pbest_loss = ctx->d_pbest_loss;
+    P.desc_pub = ctx->d_desc;
     P.ld = ctx->cfg.ld; P.N = ctx->cfg.N;
     P.q_begin = q_begin; P.q_end = q_end;
     P.tiles = ctx->tiles;
@@ -238,22 +286,21 @@ int launch_update(psops_ctx *ctx, float m, float k1, float k2, long long q_begin
     const long long span = q_end - q_begin;
     const int per_block = kUpdateThreads * (fitness ? kFitQuads : kQuads);
     const unsigned blocks = (unsigned)((span + per_block - 1) / per_block);
-    cudaError_t e;
-    if (ctx->aligned) {
-        if (fitness) e = launch_update_kernel(psops_update_kernel<true, true, kFitUnroll, kFitQuads>, blocks, stream, after_select, P);
-        else         e = launch_update_kernel(psops_update_kernel<true, false, kUnroll, kQuads>, blocks, stream, after_select, P);
-    } else {
-        if (fitness) e = launch_update_kernel(psops_update_kernel<false, true, kFitUnroll, kFitQuads>, blocks, stream, after_select, P);
-        else         e = launch_update_kernel(psops_update_kernel<false, false, kUnroll, kQuads>, blocks, stream, after_select, P);
-    }
+    const UpdateKernel kernel = pick_update_kernel(ctx->aligned, fitness, select, ctx->stream_policy);
+    if (kernel == nullptr) return PSOPS_EINVAL;
+    const cudaError_t e = launch_serialized(programmatic, kernel, dim3(blocks, 1, 1), dim3(kUpdateThreads, 1, 1), stream, P);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "psops_update_kernel launch");
+    if (select) ctx->loss_src = ctx->d_losses;      // the launch keeps a copy there
     return check_launch(ctx, "psops_update_kernel");
 }
 
 int launch_finalize(psops_ctx *ctx)
 {
-    psops_fitness_finalize_kernel<<<dim3(kFinalizeCluster, ctx->cfg.K), kFinalizeCtaThreads, 0, ctx->stream>>>(
-        ctx->d_partials, ctx->d_losses, ctx->tiles);
+    // behind the kernel that writes the tile sums; the finaliser waits for it on the device
+    const cudaError_t e = launch_serialized(true, psops_fitness_finalize_kernel, dim3(kFinalizeCluster, ctx->cfg.K),
+                                            dim3(kFinalizeCtaThreads, 1, 1), ctx->stream,
+                                            (const double *)ctx->d_partials, ctx->d_losses, ctx->tiles);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "psops_fitness_finalize_kernel launch");
     ctx->loss_src = ctx->d_losses;
     return check_launch(ctx, "psops_fitness_finalize_kernel");
 }
@@ -345,6 +392,9 @@ int psops_create(psops_ctx **out, const psops_config *cfg, float *d_x, float *d_
     ctx->d_gbest = keeps_gbest(cfg) ? (float *)(ctx->ws + lay.off_gbest) : nullptr;
     ctx->Kt = swarm_size(cfg);
     ctx->selected = false;
+    ctx->range_next = 0;
+    ctx->h_g = ctx->d_g = nullptr;
+    ctx->ev_select = nullptr;
     ctx->d_partials = (cfg->flags & PSOPS_QUADRATIC) ? (double *)(ctx->ws + lay.off_partials) : nullptr;
     ctx->dvec = ctx->tvec = nullptr;
     ctx->stream = (cudaStream_t)cuda_stream;
@@ -360,6 +410,27 @@ int psops_create(psops_ctx **out, const psops_config *cfg, float *d_x, float *d_
 
     int rc = PSOPS_OK;
     cudaError_t e = cudaGetDevice(&ctx->device);
+    // Cache policy of the streaming kernels: evict-first unless the whole state
+    // (x, v, pbest) fits in the device's L2 with room to spare, in which case
+    // the next sync finds it there.
+    ctx->stream_policy = true;
+    if (e == cudaSuccess) {
+        int l2_bytes = 0;
+        e = cudaDeviceGetAttribute(&l2_bytes, cudaDevAttrL2CacheSize, ctx->device);
+        const double state_bytes = 12.0 * (double)cfg->K * (double)cfg->N;
+        if (e == cudaSuccess && state_bytes <= (double)l2_bytes * (PSOPS_L2_RESIDENT_PERCENT / 100.0))
+            ctx->stream_policy = false;
+    }
+    // How many blocks of the single-launch form of a sync run at the same time.
+    ctx->one_wave_blocks = 0;
+    if (e == cudaSuccess && cfg->K <= 32) {
+        int sms = 0, per_sm = 0;
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device);
+        if (e == cudaSuccess)
+            e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+                &per_sm, pick_update_kernel(ctx->aligned, false, true, ctx->stream_policy), kUpdateThreads, 0);
+        ctx->one_wave_blocks = (long long)sms * per_sm;
+    }
     if (e == cudaSuccess) {
         // pBest_loss <- +inf (Algorithm 2 clones weights only), descriptor <- 0.
         std::vector<float> inf((size_t)ctx->Kt, INFINITY);
@@ -409,12 +480,22 @@ int psops_sync(psops_ctx *ctx, int64_t t_iter, float lambda)
     const float k2 = ctx->cfg.c2 / lambda;
     const bool fitness = ctx->dvec != nullptr;
 
-    rc = launch_select(ctx);
-    if (rc != PSOPS_OK) return rc;
+    // A small swarm (at most 32 particles, all blocks of the update resident at
+    // once) is launch-bound: there the update launch does the selection itself,
+    // one kernel per sync.  Anything larger, the history variant and the fused
+    // fitness run the selection kernel first and the update behind it, which
+    // costs a large grid nothing and keeps its blocks free of the closing step.
+    const long long update_blocks = (ctx->quads + (long long)kUpdateThreads * kQuads - 1) / ((long long)kUpdateThreads * kQuads);
+    const bool select_in_update = ctx->cfg.K <= 32 && !fitness && update_blocks <= ctx->one_wave_blocks &&
+                                  !(ctx->cfg.flags & (PSOPS_GBEST_HISTORY | PSOPS_SEPARATE_SELECT));
+    if (!select_in_update) {
+        rc = launch_select(ctx);
+        if (rc != PSOPS_OK) return rc;
+    }
     // With the fused fitness every warp of a tile must be whole: round the
     // quad range up to a tile; quads past the end contribute +0.0.
     const long long q_end = fitness ? ctx->tiles * 32 : ctx->quads;
-    rc = launch_update(ctx, m, k1, k2, 0, q_end, fitness, ctx->stream, /*after_select=*/true);
+    rc = launch_update(ctx, m, k1, k2, 0, q_end, fitness, ctx->stream, /*programmatic=*/true, select_in_update);
     if (rc != PSOPS_OK) return rc;
     if (fitness) {
         rc = launch_finalize(ctx);
@@ -425,39 +506,22 @@ int psops_sync(psops_ctx *ctx, int64_t t_iter, float lambda)
     return PSOPS_OK;
 }
 
-int psops_sync_host(psops_ctx *ctx, const float *h_x_in, int64_t h_in_ld, const float *h_losses,
-                    int64_t t_iter, float lambda, float *h_x_out, int64_t h_out_ld)
+// The pipelined body of psops_sync_host; any error leaves copies and kernels
+// queued, which the caller below drains before it reports the failure.
+static int sync_host_enqueue(psops_ctx *ctx, const float *h_x_in, int64_t h_in_ld, const float *h_losses,
+                             float m, float k1, float k2, bool fitness, float *h_x_out, int64_t h_out_ld)
 {
-    DeviceGuard device_guard(ctx);
-    int rc = validate_sync_args(ctx, t_iter, lambda);
-    if (rc != PSOPS_OK) return rc;
-    if (h_x_in == nullptr || h_x_out == nullptr) return PSOPS_EINVAL;
-    if (h_in_ld < ctx->cfg.N || h_out_ld < ctx->cfg.N) return PSOPS_EINVAL;
-    if (ctx->Kt != ctx->cfg.K) return PSOPS_ESTATE;
-    rc = check_host_losses(h_losses, ctx->cfg.K);
-    if (rc != PSOPS_OK) return rc;
-
     const int K = ctx->cfg.K;
     const long long N = ctx->cfg.N;
-    const float m = inertia_of(&ctx->cfg, t_iter);
-    const float k1 = ctx->cfg.c1 / lambda;
-    const float k2 = ctx->cfg.c2 / lambda;
-    const bool fitness = ctx->dvec != nullptr;
-
-    if (ctx->s_in == nullptr) {
-        PSOPS_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->s_in, cudaStreamNonBlocking));
-        PSOPS_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->s_out, cudaStreamNonBlocking));
-    }
-
     // Losses and selection first: the update of any element range needs them.
     PSOPS_CUDA(ctx, cudaMemcpyAsync(ctx->d_losses, h_losses, sizeof(float) * (size_t)K,
                                     cudaMemcpyHostToDevice, ctx->stream));
     ctx->loss_src = ctx->d_losses;
     ctx->have_losses = true;
-    rc = launch_select(ctx);
+    int rc = launch_select(ctx);
     if (rc != PSOPS_OK) return rc;
 
-    // Element ranges of whole tiles, about 32 MiB of weights per range.
+    // Element ranges of whole tiles, PSOPS_HOST_CHUNK_BYTES of weights per range.
     long long chunk_q = (((long long)PSOPS_HOST_CHUNK_BYTES) / (16ll * K)) / 32 * 32;
     if (chunk_q < 32 * 256) chunk_q = 32 * 256;
     const long long q_total = fitness ? ctx->tiles * 32 : ctx->quads;
@@ -498,10 +562,43 @@ int psops_sync_host(psops_ctx *ctx, const float *h_x_in, int64_t h_in_ld, const 
         rc = launch_finalize(ctx);
         if (rc != PSOPS_OK) return rc;
     }
+    return PSOPS_OK;
+}
+
+int psops_sync_host(psops_ctx *ctx, const float *h_x_in, int64_t h_in_ld, const float *h_losses,
+                    int64_t t_iter, float lambda, float *h_x_out, int64_t h_out_ld)
+{
+    DeviceGuard device_guard(ctx);
+    int rc = validate_sync_args(ctx, t_iter, lambda);
+    if (rc != PSOPS_OK) return rc;
+    if (h_x_in == nullptr || h_x_out == nullptr) return PSOPS_EINVAL;
+    if (h_in_ld < ctx->cfg.N || h_out_ld < ctx->cfg.N) return PSOPS_EINVAL;
+    if (ctx->Kt != ctx->cfg.K) return PSOPS_ESTATE;
+    rc = check_host_losses(h_losses, ctx->cfg.K);
+    if (rc != PSOPS_OK) return rc;
+
+    const float m = inertia_of(&ctx->cfg, t_iter);
+    const float k1 = ctx->cfg.c1 / lambda;
+    const float k2 = ctx->cfg.c2 / lambda;
+    const bool fitness = ctx->dvec != nullptr;
+
+    if (ctx->s_in == nullptr) {
+        PSOPS_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->s_in, cudaStreamNonBlocking));
+        PSOPS_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->s_out, cudaStreamNonBlocking));
+    }
+
+    rc = sync_host_enqueue(ctx, h_x_in, h_in_ld, h_losses, m, k1, k2, fitness, h_x_out, h_out_ld);
+    // Success or not, nothing may still be in flight against the caller's host
+    // buffers when this call returns: wait for both copy streams and the kernels.
+    const cudaError_t w_in = cudaStreamSynchronize(ctx->s_in);
+    const cudaError_t w_out = cudaStreamSynchronize(ctx->s_out);
+    const cudaError_t w_main = cudaStreamSynchronize(ctx->stream);
+    if (rc != PSOPS_OK) return rc;          // the state is then undefined: part of the ranges may have been updated
+    if (w_in != cudaSuccess) return cuda_fail(ctx, w_in, "psops_sync_host: input copies");
+    if (w_out != cudaSuccess) return cuda_fail(ctx, w_out, "psops_sync_host: output copies");
+    if (w_main != cudaSuccess) return cuda_fail(ctx, w_main, "psops_sync_host: kernels");
     ctx->step += 1;
     ctx->synced_once = true;
-    PSOPS_CUDA(ctx, cudaStreamSynchronize(ctx->s_out));
-    PSOPS_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     return PSOPS_OK;
 }
 
@@ -510,16 +607,36 @@ int psops_shard_select(psops_ctx *ctx, int *g)
     DeviceGuard device_guard(ctx);
     if (ctx == nullptr || g == nullptr) return PSOPS_EINVAL;
     if (!ctx->have_losses) return PSOPS_ESTATE;
-    const int rc = launch_select(ctx);
+    if (ctx->selected && ctx->range_next != 0) return PSOPS_ESTATE;     // an update is half done
+    if (ctx->h_g == nullptr) {
+        // One word of page-locked host memory that the selection kernel writes
+        // directly: the host then needs no copy and no drain of the stream, only
+        // the event behind that kernel.
+        void *host = nullptr, *dev = nullptr;
+        PSOPS_CUDA(ctx, cudaHostAlloc(&host, sizeof(int), cudaHostAllocMapped));
+        cudaError_t e = cudaHostGetDevicePointer(&dev, host, 0);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_select, cudaEventDisableTiming);
+        if (e != cudaSuccess) {
+            cudaFreeHost(host);
+            ctx->ev_select = nullptr;
+            return cuda_fail(ctx, e, "psops_shard_select: mapped word");
+        }
+        ctx->h_g = static_cast<int *>(host);
+        ctx->d_g = static_cast<int *>(dev);
+    }
+    const int rc = launch_select(ctx, ctx->d_g);
     if (rc != PSOPS_OK) return rc;
-    PSOPS_CUDA(ctx, cudaMemcpyAsync(g, &ctx->d_desc->g, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
-    PSOPS_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    PSOPS_CUDA(ctx, cudaEventRecord(ctx->ev_select, ctx->stream));
+    PSOPS_CUDA(ctx, cudaEventSynchronize(ctx->ev_select));
+    *g = *reinterpret_cast<volatile int *>(ctx->h_g);
     ctx->selected = true;
+    ctx->range_next = 0;
     ctx->synced_once = true;
     return PSOPS_OK;
 }
 
-int psops_shard_update(psops_ctx *ctx, int64_t t_iter, float lambda, const float *d_gbest_row)
+int psops_shard_update_range(psops_ctx *ctx, int64_t t_iter, float lambda, const float *d_gbest_row,
+                             int64_t first_elem, int64_t last_elem)
 {
     DeviceGuard device_guard(ctx);
     int rc = validate_sync_args(ctx, t_iter, lambda);
@@ -527,20 +644,36 @@ int psops_shard_update(psops_ctx *ctx, int64_t t_iter, float lambda, const float
     if (d_gbest_row == nullptr) return PSOPS_EINVAL;
     if (((uintptr_t)d_gbest_row & 3u) || (ctx->aligned && ((uintptr_t)d_gbest_row & 15u))) return PSOPS_EALIGN;
     if (!ctx->selected || ctx->dvec != nullptr) return PSOPS_ESTATE;
+    const long long N = ctx->cfg.N;
+    if (first_elem != ctx->range_next) return PSOPS_ESTATE;             // ranges go left to right without gaps
+    if (first_elem < 0 || last_elem <= first_elem || last_elem > N) return PSOPS_EINVAL;
+    if ((first_elem & 3) || ((last_elem & 3) && last_elem != N)) return PSOPS_EINVAL;   // whole quads
     const float m = inertia_of(&ctx->cfg, t_iter);
     const float k1 = ctx->cfg.c1 / lambda;
     const float k2 = ctx->cfg.c2 / lambda;
-    rc = launch_update(ctx, m, k1, k2, 0, ctx->quads, false, ctx->stream, false, d_gbest_row);
+    rc = launch_update(ctx, m, k1, k2, first_elem / 4, (last_elem + 3) / 4, false, ctx->stream,
+                       /*programmatic=*/false, /*select=*/false, d_gbest_row);
     if (rc != PSOPS_OK) return rc;
-    ctx->selected = false;
-    ctx->step += 1;
+    ctx->range_next = last_elem;
+    if (last_elem == N) {                   // the sync is complete
+        ctx->selected = false;
+        ctx->range_next = 0;
+        ctx->step += 1;
+    }
     return PSOPS_OK;
+}
+
+int psops_shard_update(psops_ctx *ctx, int64_t t_iter, float lambda, const float *d_gbest_row)
+{
+    if (ctx == nullptr) return PSOPS_EINVAL;
+    return psops_shard_update_range(ctx, t_iter, lambda, d_gbest_row, 0, ctx->cfg.N);
 }
 
 int psops_ssgd(psops_ctx *ctx, const float *d_grad, int64_t grad_ld, float alpha)
 {
     DeviceGuard device_guard(ctx);
     if (ctx == nullptr || d_grad == nullptr || grad_ld < ctx->cfg.N || !std::isfinite(alpha)) return PSOPS_EINVAL;
+    if (ctx->Kt != ctx->cfg.K) return PSOPS_ESTATE;     // the mean runs over the whole swarm, a shard holds a part
     if ((uintptr_t)d_grad & 3u) return PSOPS_EALIGN;
     const float scale = alpha / (float)ctx->cfg.K;
     const unsigned blocks = (unsigned)((ctx->quads + kUpdateThreads - 1) / kUpdateThreads);
@@ -615,6 +748,7 @@ int psops_average(psops_ctx *ctx)
 {
     DeviceGuard device_guard(ctx);
     if (ctx == nullptr) return PSOPS_EINVAL;
+    if (ctx->Kt != ctx->cfg.K) return PSOPS_ESTATE;     // the mean runs over the whole swarm, a shard holds a part
     const unsigned blocks = (unsigned)((ctx->quads + kUpdateThreads - 1) / kUpdateThreads);
     if (ctx->aligned)
         psops_average_kernel<true, 8><<<blocks, kUpdateThreads, 0, ctx->stream>>>(
@@ -800,6 +934,8 @@ int psops_destroy(psops_ctx *ctx)
     for (cudaEvent_t e : ctx->events) cudaEventDestroy(e);
     if (ctx->s_in) cudaStreamDestroy(ctx->s_in);
     if (ctx->s_out) cudaStreamDestroy(ctx->s_out);
+    if (ctx->ev_select) cudaEventDestroy(ctx->ev_select);
+    if (ctx->h_g) cudaFreeHost(ctx->h_g);
     delete ctx;
     return rc;
 }

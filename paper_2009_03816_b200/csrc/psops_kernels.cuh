@@ -29,7 +29,8 @@ struct SyncDesc {
     int      from_kept;         // 1: gBest of this sync is the remembered row, not row g (history mode)
     float    hist_loss;         // loss of the remembered gBest (history mode)
     int      hist_valid;        // 0 until something is remembered
-    int      pad[2];
+    unsigned int done;          // blocks of a select-in-update launch that have finished (0 between launches)
+    int      pad;
     uint32_t improved[PSOPS_MAX_K / 32];   // bit i: loss_i < pBest_loss_i
 };
 
@@ -40,6 +41,11 @@ struct UpdateParams {
     const float *dvec, *tvec;   // quadratic fitness vectors (FITNESS only)
     double *partials;           // K x tiles tile sums (FITNESS only)
     const SyncDesc *desc;
+    // Selection folded into this launch (SELECT): the K losses of this sync, the
+    // context's copy of them, pBest_loss, and the descriptor to publish into.
+    const float *loss_src;
+    float *loss_keep, *pbest_loss;
+    SyncDesc *desc_pub;
     long long ld, N;
     long long q_begin, q_end;   // quad range of this launch (quad = 4 elements)
     long long tiles;            // ceil(N / 128)
@@ -106,15 +112,20 @@ __device__ __forceinline__ float uniform24(uint32_t w)
 
 // Load / store of one quad.  nvalid = 4 on the vector path means a full
 // 128-bit access; anything else goes element by element under a bound.
-template <bool ALIGNED>
+// STREAM: evict-first accesses for a state far larger than L2 (every value is
+// touched once per sync, so keeping it only displaces the gBest row); with
+// STREAM off the accesses are ordinary write-back ones, for a state that fits
+// in L2 and is found there again by the next sync.
+template <bool ALIGNED, bool STREAM = true>
 __device__ __forceinline__ void load_quad(const float *ptr, int nvalid, float (&a)[4])
 {
     if (ALIGNED && nvalid == 4) {
-        const float4 t = __ldcs(reinterpret_cast<const float4 *>(ptr));
+        const float4 t = STREAM ? __ldcs(reinterpret_cast<const float4 *>(ptr))
+                                : *reinterpret_cast<const float4 *>(ptr);
         a[0] = t.x; a[1] = t.y; a[2] = t.z; a[3] = t.w;
     } else {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) a[e] = (e < nvalid) ? __ldcs(ptr + e) : 0.0f;
+        for (int e = 0; e < 4; ++e) a[e] = (e < nvalid) ? (STREAM ? __ldcs(ptr + e) : ptr[e]) : 0.0f;
     }
 }
 
@@ -132,15 +143,20 @@ __device__ __forceinline__ void load_quad_cached(const float *ptr, int nvalid, f
     }
 }
 
-template <bool ALIGNED>
+template <bool ALIGNED, bool STREAM = true>
 __device__ __forceinline__ void store_quad(float *ptr, int nvalid, const float (&a)[4])
 {
     if (ALIGNED && nvalid == 4) {
-        __stcs(reinterpret_cast<float4 *>(ptr), make_float4(a[0], a[1], a[2], a[3]));
+        const float4 t = make_float4(a[0], a[1], a[2], a[3]);
+        if (STREAM) __stcs(reinterpret_cast<float4 *>(ptr), t);
+        else *reinterpret_cast<float4 *>(ptr) = t;
     } else {
 #pragma unroll
         for (int e = 0; e < 4; ++e)
-            if (e < nvalid) __stcs(ptr + e, a[e]);
+            if (e < nvalid) {
+                if (STREAM) __stcs(ptr + e, a[e]);
+                else ptr[e] = a[e];
+            }
     }
 }
 
@@ -241,9 +257,25 @@ __device__ __forceinline__ bool beats(const Candidate &a, const Candidate &b)
     return a.idx < b.idx;                    // equal (or both NaN): lowest index
 }
 
+// Arg-min over one warp's candidates: after the five stages every lane holds the winner.
+__device__ __forceinline__ Candidate warp_best_candidate(Candidate c)
+{
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+        Candidate o;
+        o.loss = __shfl_xor_sync(0xffffffffu, c.loss, off);
+        o.idx = __shfl_xor_sync(0xffffffffu, c.idx, off);
+        if (beats(o, c)) c = o;
+    }
+    return c;
+}
+
+// g_host: NULL, or a word of page-locked host memory mapped into the device's
+// address space that receives g as well (particle-sharded sync: the host needs
+// g to pick the rank that broadcasts its row).
 __global__ void __launch_bounds__(PSOPS_MAX_K)
 psops_select_kernel(const float *loss, float *loss_keep, float *__restrict__ pbest_loss,
-                    SyncDesc *__restrict__ desc, int K, int history)
+                    SyncDesc *__restrict__ desc, int K, int history, int *g_host)
 {
     // Let the update kernel that follows in the stream start its prologue; it
     // waits for this grid to finish before it reads the descriptor.
@@ -267,13 +299,7 @@ psops_select_kernel(const float *loss, float *loss_keep, float *__restrict__ pbe
     c.loss = li;
     c.idx = live ? i : 0x7fffffff;
     if (!live) c.loss = __int_as_float(0x7fc00000);      // NaN with the largest index: never wins
-#pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) {
-        Candidate o;
-        o.loss = __shfl_xor_sync(0xffffffffu, c.loss, off);
-        o.idx = __shfl_xor_sync(0xffffffffu, c.idx, off);
-        if (beats(o, c)) c = o;
-    }
+    c = warp_best_candidate(c);
     if (lane == 0) warp_best[warp] = c;
     __syncthreads();
     if (i == 0) {
@@ -281,6 +307,10 @@ psops_select_kernel(const float *loss, float *loss_keep, float *__restrict__ pbe
         for (int w = 1; w < warps; ++w)
             if (beats(warp_best[w], c)) c = warp_best[w];
         desc->g = c.idx;
+        if (g_host != nullptr) {
+            *reinterpret_cast<volatile int *>(g_host) = c.idx;
+            __threadfence_system();
+        }
         // Standard-PSO variant (Section II-C, step 3): gBest from the history of
         // all particles.  The current best replaces the remembered one only on
         // a strictly smaller loss, or when nothing is remembered yet.
@@ -309,17 +339,31 @@ psops_select_kernel(const float *loss, float *loss_keep, float *__restrict__ pbe
 // loads before the first use.  Q > 1 makes every block stream a longer
 // contiguous piece of each row, which is what DRAM and the TLB like when K
 // rows x 3 arrays are all being walked at once.
+//
+// SELECT (K <= 32, whole-range launches only): the launch does the selection
+// as well, so that a sync is ONE kernel.  Every warp recomputes Algorithm 3
+// and the pBest comparisons from the K losses (K L2-served floats and a
+// five-stage shuffle), nothing is written while any block may still read the
+// old pBest_loss or step counter, and the block that finishes LAST -- known
+// from a ticket counter, no block ever waits for another -- publishes g, the
+// improved mask, the new pBest_loss and the advanced step counter.
 // ---------------------------------------------------------------------------
-template <bool ALIGNED, bool FITNESS, int U, int Q>
+template <bool ALIGNED, bool FITNESS, bool SELECT, bool STREAM, int U, int Q>
 __global__ void PSOPS_UPDATE_BOUNDS
 psops_update_kernel(const __grid_constant__ UpdateParams P)
 {
+    static_assert(!(SELECT && FITNESS), "the single-launch form carries no fitness");
     const long long q0 = P.q_begin + (long long)blockIdx.x * (kUpdateThreads * Q) + threadIdx.x;
-    // Launched with programmatic stream serialisation right behind the selection
-    // kernel: everything that kernel wrote is visible after this wait (a no-op
-    // for an ordinary launch).
+    // Whatever follows in the stream with programmatic serialisation (the
+    // fitness finaliser, the next sync) may be made resident now; it waits for
+    // this grid to finish before it reads anything.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // Launched with programmatic stream serialisation behind the kernel in
+    // front of it: everything that kernel wrote is visible after this wait (a
+    // no-op for an ordinary launch).
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (!FITNESS && q0 >= P.q_end) return;   // with FITNESS whole warps stay for the shuffles
+    if (!FITNESS && !SELECT && q0 >= P.q_end) return;   // with FITNESS whole warps stay for the shuffles,
+                                                        // with SELECT whole blocks for the closing barrier
 
     bool active[Q];
     int nvalid[Q];
@@ -333,21 +377,46 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
         if (active[j] && d0 < P.N) nvalid[j] = (P.N - d0 >= 4) ? 4 : (int)(P.N - d0);
         col[j] = (size_t)d0;
     }
+    const int lane = threadIdx.x & 31;
+
+    // Selection results: read from the descriptor the selection kernel filled,
+    // or (SELECT) recomputed here by every warp; lane i stands for particle i.
+    uint32_t step;
+    int g;
+    int from_kept = 0;
+    uint32_t sel_word = 0;                   // SELECT: improved bits of particles 0..31
+    float sel_loss = 0.0f;
+    bool sel_improved = false;
+    if (SELECT) {
+        const bool live = lane < P.K;
+        sel_loss = live ? __ldcg(P.loss_src + lane) : 0.0f;
+        const float pl = live ? __ldcg(P.pbest_loss + lane) : 0.0f;
+        sel_improved = live && (sel_loss < pl);          // strict: an equal loss never replaces pBest
+        sel_word = __ballot_sync(0xffffffffu, sel_improved);
+        Candidate c;
+        c.loss = live ? sel_loss : __int_as_float(0x7fc00000);
+        c.idx = live ? lane : 0x7fffffff;
+        g = warp_best_candidate(c).idx;
+        step = __ldcg(&P.desc_pub->next_step);
+    } else {
+        step = P.desc->step;
+        g = P.desc->g;
+        from_kept = P.desc->from_kept;
+    }
 
     // gBest = row g as it is BEFORE this sync overwrites it; this thread is the
     // only writer of these elements, so reading them first is enough.
     // It comes from row g of this context, from the remembered row (history
     // mode, when the current best did not beat it) or from a row handed in by
     // the caller (sharded swarm).
-    const uint32_t step = P.desc->step;
     const float *gsrc = P.gbest_ext;
-    bool keep_copy = false;
+    bool keep_copy = P.gbest_copy != nullptr;
     if (gsrc == nullptr) {
-        if (P.desc->from_kept) {
+        if (from_kept) {
             gsrc = P.gbest_copy;
+            keep_copy = false;               // it is the copy
         } else {
-            gsrc = P.x + (size_t)P.desc->g * (size_t)P.ld;
-            keep_copy = P.gbest_copy != nullptr;
+            gsrc = P.x + (size_t)g * (size_t)P.ld;
         }
     }
     float gb[Q][4];
@@ -355,7 +424,7 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
 #pragma unroll
     for (int j = 0; j < Q; ++j) {
         load_quad_cached<ALIGNED>(gsrc + col[j], nvalid[j], gb[j]);
-        if (keep_copy) store_quad<ALIGNED>(P.gbest_copy + col[j], nvalid[j], gb[j]);
+        if (keep_copy) store_quad<ALIGNED, STREAM>(P.gbest_copy + col[j], nvalid[j], gb[j]);
         if (FITNESS) {
             load_quad_cached<ALIGNED>(P.dvec + col[j], nvalid[j], dv[j]);
             load_quad_cached<ALIGNED>(P.tvec + col[j], nvalid[j], tv[j]);
@@ -371,7 +440,6 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
     // issued, so that the shuffle chain sits in the shadow of the loads.
     double fq[Q][U];                         // level-0 fitness sums of the previous batch
     int fq_i0 = -1;
-    const int lane = threadIdx.x & 31;
     auto flush_fitness = [&]() {
 #pragma unroll
         for (int j = 0; j < Q; ++j) {
@@ -383,9 +451,9 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
     };
 
     size_t row = 0;                          // offset of row i0
-    uint32_t impw = 0;                       // improved bits of particles i0 - i0 % 32 .. +31 (local numbering)
+    uint32_t impw = sel_word;                // improved bits of particles i0 - i0 % 32 .. +31 (local numbering)
     for (int i0 = 0; i0 < P.K; i0 += U) {
-        if ((i0 & 31) == 0) {
+        if (!SELECT && (i0 & 31) == 0) {
             // One window of 32 bits per 32 particles, fetched ahead of the loads it
             // steers: a per-particle fetch would sit between them and stall the
             // in-order issue.  The window starts at swarm-wide particle i_first + i0.
@@ -405,9 +473,9 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
 #pragma unroll
                 for (int j = 0; j < Q; ++j) {
                     const size_t at = row + (size_t)u * (size_t)P.ld + col[j];
-                    load_quad<ALIGNED>(P.x + at, nvalid[j], xo[u][j]);
-                    load_quad<ALIGNED>(P.v + at, nvalid[j], vo[u][j]);
-                    if (!imp[u]) load_quad<ALIGNED>(P.p + at, nvalid[j], pp[u][j]);
+                    load_quad<ALIGNED, STREAM>(P.x + at, nvalid[j], xo[u][j]);
+                    load_quad<ALIGNED, STREAM>(P.v + at, nvalid[j], vo[u][j]);
+                    if (!imp[u]) load_quad<ALIGNED, STREAM>(P.p + at, nvalid[j], pp[u][j]);
                 }
             }
         }
@@ -445,9 +513,9 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
                         vn[e] = __fmaf_rn(t2, dg, __fmaf_rn(t1, dl, a0));  // Eq. 6
                         xn[e] = __fadd_rn(w, vn[e]);                        // Eq. 7
                     }
-                    store_quad<ALIGNED>(P.v + at, nvalid[j], vn);
-                    store_quad<ALIGNED>(P.x + at, nvalid[j], xn);
-                    if (imp[u]) store_quad<ALIGNED>(P.p + at, nvalid[j], xo[u][j]);
+                    store_quad<ALIGNED, STREAM>(P.v + at, nvalid[j], vn);
+                    store_quad<ALIGNED, STREAM>(P.x + at, nvalid[j], xn);
+                    if (imp[u]) store_quad<ALIGNED, STREAM>(P.p + at, nvalid[j], xo[u][j]);
                     if (FITNESS) fq[j][u] = fitness_quad_sum(xn, dv[j], tv[j], nvalid[j]);
                 }
             }
@@ -455,6 +523,38 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
         row += (size_t)U * (size_t)P.ld;
     }
     if (FITNESS && fq_i0 >= 0) flush_fitness();
+
+    if (SELECT) {
+        // Every warp of this block read the old selection state before this
+        // barrier; the ticket is taken after it.  The block that draws the last
+        // ticket therefore knows that no block will read that state again, and
+        // it alone moves it on.  Nobody waits: a block that is not last leaves.
+        __syncthreads();
+        if (threadIdx.x < 32) {
+            unsigned int ticket = 0;
+            if (lane == 0) {
+                __threadfence();
+                ticket = atomicAdd(&P.desc_pub->done, 1u);
+            }
+            ticket = __shfl_sync(0xffffffffu, ticket, 0);
+            if (ticket == gridDim.x - 1) {
+                __threadfence();
+                if (lane < P.K) {
+                    P.loss_keep[lane] = sel_loss;                 // the context's own copy of the losses
+                    if (sel_improved) P.pbest_loss[lane] = sel_loss;
+                }
+                if (lane == 0) {
+                    SyncDesc *d = P.desc_pub;
+                    d->g = g;
+                    d->improved[0] = sel_word;
+                    d->from_kept = 0;
+                    d->step = step;
+                    d->next_step = step + 1u;
+                    d->done = 0u;
+                }
+            }
+        }
+    }
 }
 
 // ---------------------------------------------------------------------------
@@ -540,6 +640,8 @@ psops_fitness_tiles_kernel(const float *__restrict__ x, const float *__restrict_
     const long long q = (long long)blockIdx.x * kUpdateThreads + threadIdx.x;
     const long long d0 = q * 4;
     int nvalid = 0;
+    // the finaliser behind this kernel may be made resident; it waits for this grid
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (q < quads) nvalid = (N - d0 >= 4) ? 4 : (int)(N - d0);
     if ((q >> 5) >= tiles) return;           // whole warp out of range
     float dv[4], tv[4];
@@ -568,7 +670,9 @@ psops_fitness_tiles_kernel(const float *__restrict__ x, const float *__restrict_
 // tau + 1024, ... in increasing order (loads run ahead, the additions stay a
 // chain), each warp butterflies its group, and the 32 group sums meet in the
 // shared memory of the cluster's first block, whose first thread adds them in
-// group order.  cluster.sync() is the hardware cluster barrier.
+// group order.  cluster.sync() is the hardware cluster barrier; the
+// arrive/wait pair in front of the remote store is the same barrier, split so
+// that the wait comes after the loads.
 #ifndef PSOPS_FINALIZE_DEPTH
 #define PSOPS_FINALIZE_DEPTH 32        // tile sums in flight per thread of the finaliser
 #endif
@@ -587,6 +691,13 @@ psops_fitness_finalize_kernel(const double *__restrict__ partials, float *__rest
     const int i = blockIdx.y;
     const int tau = (int)rank * kFinalizeCtaThreads + (int)threadIdx.x;      // slot
     const double *row = partials + (size_t)i * (size_t)tiles;
+    // Another block's shared memory may only be touched once that block is
+    // running: every block arrives at the cluster barrier here and waits for
+    // the others just before the remote store, after its own loads.
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    // Launched with programmatic stream serialisation behind the kernel that
+    // writes the tile sums: they are visible after this wait.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     double acc = 0.0;
     // Only 1024 chains per particle exist, so each thread keeps many loads in
@@ -606,6 +717,7 @@ psops_fitness_finalize_kernel(const double *__restrict__ partials, float *__rest
 #pragma unroll
     for (int off = 16; off >= 1; off >>= 1)
         acc = __dadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, off));
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");      // all blocks of the cluster run
     if ((threadIdx.x & 31) == 0) {
         double *first = cluster.map_shared_rank(group, 0);
         first[tau >> 5] = acc;

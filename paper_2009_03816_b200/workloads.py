@@ -180,3 +180,21 @@ def sample_columns(N: int, count: int, seed: int) -> np.ndarray:
     edge = np.concatenate([np.arange(min(8, N)), np.arange(max(0, N - 8), N)])
     rnd = np.random.default_rng([seed, 99]).integers(0, N, size=max(0, count))
     return np.unique(np.concatenate([edge, rnd]).astype(np.int64))
+
+
+def sample_columns_dense(N: int, count: int, seed: int, block: int = 1024) -> np.ndarray:
+    """A larger sample for full-size checks: `count` seeded random elements,
+    plus one element of every residue modulo `block` (the elements one thread
+    block of the update kernel covers) in a seeded random block, plus the first
+    and last element of the first, a middle and the last block, plus the
+    vector's head and ragged tail."""
+    rng = np.random.default_rng([seed, 98])
+    blocks = (N + block - 1) // block
+    residues = np.arange(block, dtype=np.int64) + block * rng.integers(0, max(1, blocks - 1), size=block)
+    edges = []
+    for b in (0, blocks // 2, blocks - 1):
+        edges += [b * block, min(N, (b + 1) * block) - 1]
+    head_tail = np.concatenate([np.arange(min(8, N)), np.arange(max(0, N - 8), N)])
+    rnd = rng.integers(0, N, size=max(0, count))
+    cols = np.concatenate([residues, np.asarray(edges, dtype=np.int64), head_tail, rnd]).astype(np.int64)
+    return np.unique(cols[(cols >= 0) & (cols < N)])

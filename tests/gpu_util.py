@@ -27,6 +27,9 @@ def assert_close(got, want, what=""):
     got = np.asarray(got)
     want = np.asarray(want)
     assert got.shape == want.shape, (what, got.shape, want.shape)
+    if got.dtype == np.float32 and want.dtype == np.float32 and got.flags.c_contiguous and want.flags.c_contiguous \
+            and np.array_equal(got.view(np.uint32), want.view(np.uint32)):
+        return 0                                          # identical bits: nothing more to look at
     rms = float(np.sqrt(np.mean(want.astype(np.float64) ** 2))) if want.size else 0.0
     tol = 1e-6 * np.maximum(np.abs(want).astype(np.float64), 1e-6 * rms)
     diff = np.abs(got.astype(np.float64) - want.astype(np.float64))
@@ -39,6 +42,35 @@ def assert_close(got, want, what=""):
             f"gpu={got[tuple(idx)]!r} ref={want[tuple(idx)]!r}")
     same = (got.view(np.uint32) == want.view(np.uint32)) | ((got == 0) & (want == 0))
     return int(got.size - same.sum())
+
+
+def device_compare(dev_rows, want, what="", rows_per_piece=4):
+    """The same contract for a whole swarm without bringing it to the host: the
+    oracle's rows are uploaded piece by piece and compared on the device (plain
+    torch comparisons; this is the checker, not the path).  Returns the number of
+    elements that are not bit-identical (+0 and -0 count as identical); raises if
+    any element is outside |gpu - ref| <= 1e-6 * max(|ref|, 1e-6 * RMS(ref))."""
+    K, n = want.shape
+    assert tuple(dev_rows.shape) == (K, n), (what, tuple(dev_rows.shape), want.shape)
+    rms = float(np.sqrt(np.mean(np.square(want, dtype=np.float64))))
+    inexact = 0
+    for k0 in range(0, K, rows_per_piece):
+        ref = torch.from_numpy(np.ascontiguousarray(want[k0:k0 + rows_per_piece])).to(dev_rows.device)
+        got = dev_rows[k0:k0 + rows_per_piece]
+        differ = (got.view(torch.int32) != ref.view(torch.int32)) & ~((got == 0) & (ref == 0))
+        n_differ = int(differ.sum().item())
+        if n_differ:
+            tol = 1e-6 * torch.clamp(ref.abs().double(), min=1e-6 * rms)
+            outside = ~((got.double() - ref.double()).abs() <= tol) & differ
+            n_out = int(outside.sum().item())
+            if n_out:
+                idx = torch.nonzero(outside)[0].tolist()
+                raise AssertionError(
+                    f"{what}: {n_out} elements of rows {k0}.. outside 1e-6; first at "
+                    f"({k0 + idx[0]}, {idx[1]}): gpu={got[idx[0], idx[1]].item()!r} ref={ref[idx[0], idx[1]].item()!r}")
+        inexact += n_differ
+        del ref, differ
+    return inexact
 
 
 class DeviceRows:

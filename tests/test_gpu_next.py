@@ -148,6 +148,75 @@ def test_particle_shards_reproduce_the_unsharded_sync(counts):
         sw.close()
 
 
+def test_shards_update_in_ranges_owner_reads_its_own_row_and_gbest_is_kept():
+    """The multi-GPU driver's calls, shard after shard on one GPU: the update
+    goes over the element ranges of a chunked broadcast; the shard that holds
+    gBest reads the row in place from its own weights; with PSOPS_KEEP_GBEST
+    every shard keeps a copy of the row it was given."""
+    counts = [3, 1, 4]
+    K, N = sum(counts), 50_003
+    ld = (N + 1023) // 1024 * 1024
+    x, v, p = _swarm(K, N, 12)
+    gpu_util.ensure_library()
+    ref = oracle.RefSwarm(x, v, p, m_max=0.9, m_min=0.3, t_max=40, c1=0.2, c2=0.9, seed=5, nthreads=NTHREADS)
+    shards, first = [], 0
+    for n in counts:
+        rows = [gpu_util.DeviceRows(a[first:first + n], N, ld) for a in (x, v, p)]
+        sw = binding.Swarm(rows[0].rows, rows[1].rows, rows[2].rows, N=N, m_max=0.9, m_min=0.3, t_max=40,
+                           c1=0.2, c2=0.9, seed=5, k_first=first, K_total=K, flags=binding.PSOPS_KEEP_GBEST)
+        shards.append((first, n, rows, sw))
+        first += n
+    bounds = sharded.range_bounds(N, 4)
+    assert len(bounds) == 4 and bounds[-1][1] == N and N % 4 == 3
+    received = torch.zeros(N, device="cuda")           # what a broadcast would deliver to the other shards
+    rng = np.random.default_rng(2)
+    for s in range(5):
+        loss = rng.random(K).astype(np.float32)
+        loss[[2, 3, 6, 0, 5][s]] = 0.0                 # gBest on every shard in turn, first and last rows too
+        dl = torch.from_numpy(loss).cuda()
+        gs = [sw.set_losses(dl) or sw.shard_select() for _, _, _, sw in shards]
+        assert len(set(gs)) == 1
+        owner, row = sharded.owner_of(gs[0], counts)
+        received.copy_(shards[owner][3].x[row, :N])    # leaves the owner before anything is overwritten
+        for r, (_, _, _, sw) in enumerate(shards):
+            src = sw.x[row, :N] if r == owner else received
+            for a, b in bounds:
+                sw.shard_update_range(src, a, b, 4 * s, 1.0 + s)
+        ref.sync(loss, 4 * s, 1.0 + s, want_gbest=True)
+        assert gs[0] == ref.g
+        for f, n, rows, sw in shards:
+            g, improved, pl = sw.info()
+            assert np.array_equal(improved, ref.improved) and np.array_equal(pl, ref.pbest_loss)
+            assert np.array_equal(sw.row(PSOPS_GBEST), ref.gbest)
+            for d, want, name in zip(rows, (ref.x, ref.v, ref.p), "xvp"):
+                assert assert_close(d.host(), want[f:f + n], f"shard@{f} s={s} {name}") == 0
+    _, _, rows, sw = shards[0]
+    # ranges must come left to right, on quad boundaries, after a selection
+    sw.set_losses(dl)
+    sw.shard_select()
+    for a, b, code in ((4, 8, binding.PSOPS_ESTATE), (0, 6, binding.PSOPS_EINVAL), (0, N + 1, binding.PSOPS_EINVAL)):
+        with pytest.raises(binding.PsopsError) as e:
+            sw.shard_update_range(received, a, b)
+        assert e.value.code == code
+    sw.shard_update_range(received, 0, 1024)
+    with pytest.raises(binding.PsopsError) as e:
+        sw.shard_select()                                # an update is half done
+    assert e.value.code == binding.PSOPS_ESTATE
+    with pytest.raises(binding.PsopsError) as e:
+        sw.shard_update_range(received, 0, 1024)         # the same range again
+    assert e.value.code == binding.PSOPS_ESTATE
+    sw.shard_update_range(received, 1024, N)
+    # the whole-swarm operations are refused on a shard
+    for fn in (sw.average, lambda: sw.ssgd(rows[0].rows, -0.1)):
+        with pytest.raises(binding.PsopsError) as e:
+            fn()
+        assert e.value.code == binding.PSOPS_ESTATE
+    for _, _, rows, sw in shards:
+        for d in rows:
+            d.check_canaries("shard ranges")
+        sw.close()
+
+
 def test_sharded_driver_single_rank():
     """The driver class on one rank (no process group): same calls, same result."""
     K, N = 4, 5000

@@ -11,7 +11,7 @@ import torch
 import oracle
 from paper_2009_03816_b200 import binding, workloads
 from paper_2009_03816_b200.binding import (PSOPS_GBEST, PSOPS_KEEP_GBEST, PSOPS_PBEST,
-                                           PSOPS_QUADRATIC, PSOPS_V, PSOPS_X)
+                                           PSOPS_QUADRATIC, PSOPS_SEPARATE_SELECT, PSOPS_V, PSOPS_X)
 
 import gpu_util
 from gpu_util import NTHREADS, Pair, assert_close
@@ -32,9 +32,16 @@ def _swarm(K, N, seed, sv=0.1):
 # ---------------------------------------------------------------------------
 @pytest.mark.parametrize("N", [1, 2, 3, 5, 127, 128, 129, 1000, 4099])
 @pytest.mark.parametrize("K", [1, 2, 3, 32, 33])
-def test_small_shapes_vector_path(K, N):
+@pytest.mark.parametrize("separate", [False, True], ids=["one_launch", "select_kernel"])
+def test_small_shapes_vector_path(K, N, separate):
+    """Up to 32 particles a sync is one launch that selects and updates;
+    PSOPS_SEPARATE_SELECT (and any larger swarm) runs the selection kernel
+    first.  Both must follow the oracle bit for bit."""
+    if separate and K > 32:
+        pytest.skip("more than 32 particles always use the selection kernel")
     x, v, p = _swarm(K, N, 100 * K + N)
-    pair = Pair(x, v, p, N, m_max=0.9, m_min=0.3, t_max=10, c1=0.2, c2=0.9, seed=K * 7919 + N)
+    pair = Pair(x, v, p, N, m_max=0.9, m_min=0.3, t_max=10, c1=0.2, c2=0.9, seed=K * 7919 + N,
+                flags=PSOPS_SEPARATE_SELECT if separate else 0)
     rng = np.random.default_rng(N)
     for s in range(4):
         pair.sync(rng.random(K).astype(np.float32), t=3 * s, lam=1.0 + s)
@@ -42,6 +49,7 @@ def test_small_shapes_vector_path(K, N):
         pair.check_state(f"K={K} N={N} s={s}")
     pair.check_canaries()
     assert pair.inexact == 0          # same rounding sequence on both sides
+    assert pair.gpu.launches == (8 if separate or K > 32 else 4)
     pair.close()
 
 
@@ -78,8 +86,9 @@ def test_many_particles():
 # ---------------------------------------------------------------------------
 # Selection edge cases through the device kernel.
 # ---------------------------------------------------------------------------
-def test_selection_ties_nan_inf_on_device():
-    K, N = 40, 64
+@pytest.mark.parametrize("K", [20, 32, 40])          # selection inside the update launch / selection kernel
+def test_selection_ties_nan_inf_on_device(K):
+    N = 64
     x, v, p = _swarm(K, N, 9)
     pair = Pair(x, v, p, N, m_max=0.7, m_min=0.7, c1=1.5, c2=1.5, seed=3)
     rng = np.random.default_rng(1)
@@ -88,20 +97,20 @@ def test_selection_ties_nan_inf_on_device():
         loss = rng.integers(0, 3, size=K).astype(np.float32)
         cases.append(loss)
     cases.append(np.full(K, np.inf, np.float32))
-    cases.append(np.where(np.arange(K) == 37, -0.0, 0.0).astype(np.float32))
+    cases.append(np.where(np.arange(K) == K - 3, -0.0, 0.0).astype(np.float32))
     for loss in cases:
         pair.sync(loss)
         pair.check_selection()
     # device-side NaN losses (the host path refuses them): they never win
     dl = np.full(K, np.nan, np.float32)
-    dl[35] = 5.0
-    dl[36] = 5.0
+    dl[K - 5] = 5.0
+    dl[K - 4] = 5.0
     dev = torch.from_numpy(dl).cuda()
     pair.gpu.set_losses(dev)
     pair.gpu.sync()
     pair.ref.sync(dl)
     pair.check_selection()
-    assert pair.ref.g == 35
+    assert pair.ref.g == K - 5
     dev = torch.from_numpy(np.full(K, np.nan, np.float32)).cuda()
     pair.gpu.set_losses(dev)
     pair.gpu.sync()
@@ -166,10 +175,14 @@ def test_cfg4_scaled():
 
 
 def _run_sampled(w, count):
-    """Full-size run on the GPU; the oracle follows a sample of columns (every
-    element is independent of the others once the losses are given)."""
+    """Full-size run on the GPU in the launch configuration the benchmark times
+    (device-resident loss table); the oracle follows a sample of columns (every
+    element is independent of the others once the losses are given): `count`
+    random ones, every residue of the element index modulo a thread block's
+    1024 elements, block edges, the vector's head and ragged tail."""
     gpu_util.ensure_library()
-    cols = workloads.sample_columns(w.N, count, w.seed)
+    cols = workloads.sample_columns_dense(w.N, count, w.seed)
+    assert cols.size >= count * 0.95 and set((cols % 1024).tolist()) == set(range(1024))
     dev = torch.device("cuda:0")
     dx = torch.zeros((w.K, w.ld), dtype=torch.float32, device=dev)
     dv = torch.zeros((w.K, w.ld), dtype=torch.float32, device=dev)
@@ -186,7 +199,7 @@ def _run_sampled(w, count):
     table = workloads.losses(w)
     gpu = binding.Swarm(dx, dv, dp, N=w.N, m_max=w.omega, m_min=w.omega, c1=w.c1, c2=w.c2, seed=w.seed)
     ref = oracle.RefSwarm(xs, vs, xs, m_max=w.omega, m_min=w.omega, t_max=1, c1=w.c1, c2=w.c2,
-                          seed=w.seed, elem_index=cols)
+                          seed=w.seed, elem_index=cols, nthreads=NTHREADS)
     dtable = torch.from_numpy(table).to(dev)
     dcols = torch.from_numpy(cols).to(dev)
     inexact = 0
@@ -207,11 +220,57 @@ def _run_sampled(w, count):
 
 
 def test_cfg3_full_size_sampled():
-    assert _run_sampled(workloads.CONFIGS["cfg3"], 4000) == 0
+    assert _run_sampled(workloads.CONFIGS["cfg3"], 200_000) == 0
 
 
 def test_cfg4_full_size_sampled():
-    assert _run_sampled(workloads.CONFIGS["cfg4"], 2000) == 0
+    w = workloads.CONFIGS["cfg4"]
+    assert workloads.sample_columns_dense(w.N, 1_050_000, w.seed).size >= 1_000_000
+    assert _run_sampled(w, 1_050_000) == 0
+
+
+def _run_whole_swarm(w, syncs, checkpoints):
+    """Full size on both sides: the oracle carries the whole swarm (all host
+    cores), selection is compared after every sync and EVERY element of x, v
+    and pbest at the checkpoints and after the last sync.  Elements never
+    interact, so a wrong element at any sync is still wrong at the end."""
+    gpu_util.ensure_library()
+    dev = torch.device("cuda:0")
+    x, v, p = workloads.state(w)
+    dx, dv = torch.from_numpy(x).to(dev), torch.from_numpy(v).to(dev)
+    dp = dx.clone()
+    ref = oracle.RefSwarm(x[:, :w.N], v[:, :w.N], p[:, :w.N], m_max=w.omega, m_min=w.omega, t_max=1,
+                          c1=w.c1, c2=w.c2, seed=w.seed, nthreads=NTHREADS)
+    del x, v, p
+    table = workloads.losses(w)
+    dtable = torch.from_numpy(table).to(dev)
+    gpu = binding.Swarm(dx, dv, dp, N=w.N, m_max=w.omega, m_min=w.omega, c1=w.c1, c2=w.c2, seed=w.seed)
+    inexact = 0
+    for s in range(syncs):
+        gpu.set_losses(dtable[s])
+        gpu.sync(0, w.lam)
+        ref.sync(table[s], 0, w.lam)
+        g, improved, pl = gpu.info()
+        assert g == ref.g and np.array_equal(improved, ref.improved), s
+        assert np.array_equal(pl.view(np.uint32), ref.pbest_loss.view(np.uint32)), s
+        if s in checkpoints or s == syncs - 1:
+            for name, t, want in (("x", dx, ref.x), ("v", dv, ref.v), ("pbest", dp, ref.p)):
+                inexact += gpu_util.device_compare(t[:, :w.N], want, f"{w.name} s={s} {name}")
+    assert torch.all(dx[:, w.N:] == 0) and torch.all(dv[:, w.N:] == 0) and torch.all(dp[:, w.N:] == 0)
+    gpu.close()
+    return inexact
+
+
+def test_cfg3_full_size_whole_swarm_all_syncs():
+    w = workloads.CONFIGS["cfg3"]
+    assert _run_whole_swarm(w, w.S, checkpoints=(0, 9, 49)) == 0
+
+
+def test_cfg4_full_size_whole_swarm_first_syncs():
+    import psutil
+    if psutil.virtual_memory().available < (40 << 30):
+        pytest.skip("the oracle's copy of the 9.8 GB swarm plus the generator's needs about 30 GB of host memory")
+    assert _run_whole_swarm(workloads.CONFIGS["cfg4"], 3, checkpoints=(0,)) == 0
 
 
 # ---------------------------------------------------------------------------
@@ -235,6 +294,36 @@ def test_quadratic_fitness_standalone_bit_exact(N):
     got = pair.gpu.losses()
     want = oracle.quadratic_losses(pair.ref.x, d, t, nthreads=NTHREADS)
     assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+    pair.close()
+
+
+def _fitness_order_cases():
+    import golden_cases
+    return golden_cases.fitness_order_cases()
+
+
+@pytest.mark.parametrize("case", _fitness_order_cases(), ids=lambda c: c[0])
+def test_quadratic_fitness_hand_worked_order_on_device(case):
+    """The hand-worked cancellation cases that fix the summation order and the
+    term rounding, through the stand-alone fitness kernels and through the
+    fitness fused into the update (pure inertia, v = 0: the new weights equal
+    the old ones exactly, so the fused pass sees the same rows)."""
+    name, w, d, t, want = case
+    n = w.size
+    x = np.stack([w, t, w])                              # row 1 sits at the minimiser: fitness 0
+    zeros = np.zeros_like(x)
+    pair = Pair(x, zeros, x, n, m_max=1.0, m_min=1.0, c1=0.0, c2=0.0, seed=1, flags=PSOPS_QUADRATIC)
+    dd, dt = torch.from_numpy(d).cuda(), torch.from_numpy(t).cuda()
+    pair.gpu.set_quadratic(dd, dt)
+    pair.gpu.eval_quadratic()
+    got = pair.gpu.losses()
+    assert got[0].view(np.uint32) == want.view(np.uint32), (name, float(got[0]), float(want))
+    assert got[2].view(np.uint32) == want.view(np.uint32) and got[1] == 0.0
+    pair.gpu.sync()                                      # x' = x + 1 * 0 exactly; losses of x' from the fused pass
+    fused = pair.gpu.losses()
+    assert np.array_equal(pair.dx.host(), x)
+    assert fused[0].view(np.uint32) == want.view(np.uint32), (name, float(fused[0]), float(want))
+    assert fused[2].view(np.uint32) == want.view(np.uint32) and fused[1] == 0.0
     pair.close()
 
 
@@ -283,9 +372,11 @@ def test_cfg5_scalar_path_fused_fitness():
 
 def test_cfg5_full_size(syncs=None):
     """Full 50 M-element vectors, fitness fused into the update; the oracle
-    runs the whole swarm on all host cores for a bounded number of syncs
-    (PSOPS_CFG5_SYNCS=200 runs the whole recipe, about 2.5 minutes)."""
-    syncs = int(os.environ.get("PSOPS_CFG5_SYNCS", "6")) if syncs is None else syncs
+    runs the whole swarm on all host cores.  All 200 syncs of the recipe by
+    default (PSOPS_CFG5_SYNCS shortens the run for a quick look): losses bit-exact
+    and selection identical after every sync, every element of x, v, pbest at
+    three checkpoints and at the end."""
+    syncs = int(os.environ.get("PSOPS_CFG5_SYNCS", "200")) if syncs is None else syncs
     w = workloads.CONFIGS["cfg5"]
     gpu_util.ensure_library()
     dev = torch.device("cuda:0")
@@ -302,18 +393,18 @@ def test_cfg5_full_size(syncs=None):
                           c1=w.c1, c2=w.c2, seed=w.seed, nthreads=NTHREADS)
     del x, v, p
     loss = oracle.quadratic_losses(ref.x, d, t, nthreads=NTHREADS)
-    cols = torch.from_numpy(workloads.sample_columns(w.N, 200_000, 5)).to(dev)
     for s in range(syncs):
         assert np.array_equal(gpu.losses().view(np.uint32), loss.view(np.uint32)), s
         gpu.sync(0, w.lam)
         ref.sync(loss, 0, w.lam)
         g, improved, pl = gpu.info()
-        assert g == ref.g and np.array_equal(improved, ref.improved)
+        assert g == ref.g and np.array_equal(improved, ref.improved), s
+        assert np.array_equal(pl.view(np.uint32), ref.pbest_loss.view(np.uint32)), s
         loss = oracle.quadratic_losses(ref.x, d, t, nthreads=NTHREADS)
+        if s in (0, 19, 99) or s == syncs - 1:
+            for name, tdev, want in (("x", dx, ref.x), ("v", dv, ref.v), ("pbest", dp, ref.p)):
+                assert gpu_util.device_compare(tdev[:, :w.N], want, f"cfg5 s={s} {name}") == 0
     assert np.array_equal(gpu.losses().view(np.uint32), loss.view(np.uint32))
-    hc = cols.cpu().numpy()
-    for name, tdev, want in (("x", dx, ref.x), ("v", dv, ref.v), ("pbest", dp, ref.p)):
-        assert assert_close(tdev[:, cols].cpu().numpy(), want[:, hc], name) == 0
     gpu.close()
 
 
@@ -476,10 +567,16 @@ def test_runs_on_a_side_stream_and_counts_launches():
     sw.sync()
     ref.sync(loss)
     stream.synchronize()
-    assert sw.launches == 2                        # selection + fused update
+    assert sw.launches == 1                        # four particles: selection and update are one launch
     assert assert_close(t[0].cpu().numpy(), ref.x) == 0
     sw.average()
-    assert sw.launches == 3
+    assert sw.launches == 2
+    sw.close()
+    sw = binding.Swarm(*t, N=N, m_max=0.7, m_min=0.7, c1=1.5, c2=1.5, seed=8, stream=stream.cuda_stream,
+                       flags=PSOPS_SEPARATE_SELECT)
+    sw.set_losses(loss)
+    sw.sync()
+    assert sw.launches == 2                        # selection kernel + update kernel
     sw.close()
 
 

@@ -51,7 +51,7 @@ def test_workspace_bytes(lib):
                                flags=binding.PSOPS_QUADRATIC)
     assert binding.psops_workspace_bytes(quad) >= n0 + 8 * 8 * 8      # K x ceil(N/128) doubles
     for bad in (dict(K=0), dict(K=1025), dict(N=0), dict(N=1 << 33), dict(ld=999), dict(t_max=0),
-                dict(flags=8), dict(c1=float("nan")), dict(m_max=float("inf"))):
+                dict(flags=16), dict(c1=float("nan")), dict(m_max=float("inf"))):
         kw = dict(K=8, N=1000, ld=1000, m_max=0.7, m_min=0.7, t_max=1, c1=1.5, c2=1.5, seed=1, flags=0)
         kw.update(bad)
         K, N, ld = kw.pop("K"), kw.pop("N"), kw.pop("ld")

@@ -91,26 +91,30 @@ SHARD_WORKER = textwrap.dedent("""
     first = sharded.first_index(r.rank, counts)
 
     class Engine:                       # holds only this rank's rows of the reference swarm
-        def __init__(self): self.got = None; self.log = []
+        def __init__(self): self.log = []
         def set_losses(self, all_losses): self.losses = all_losses.numpy().copy()
-        def shard_select(self): return oracle.argmin(self.losses)
-        def copy_row(self, row, out):
-            self.log.append(("copy", row)); out.copy_(torch.from_numpy(full.x[first + row]))
-        def shard_update(self, gbest, t, lam):
-            pre = full.x.copy()
-            full.sync(self.losses, t, lam, want_gbest=True)
-            assert np.array_equal(gbest.numpy(), full.gbest), "broadcast row is not gBest"
-            assert np.array_equal(gbest.numpy(), pre[full.g])
+        def shard_select(self):
+            self.g = oracle.argmin(self.losses); self.pre = full.x.copy(); return self.g
+        def row(self, row):             # the owner sends this memory itself, nothing is copied out
+            self.log.append(("row", row)); return torch.from_numpy(full.x[first + row])
+        def shard_update_range(self, gbest, a, b, t, lam):
+            self.log.append(("range", a, b))
+            assert np.array_equal(gbest.numpy()[a:b], self.pre[self.g][a:b]), "range has not arrived"
+            if b == N:                  # last range: the whole row is here; now the weights may change
+                assert np.array_equal(gbest.numpy(), self.pre[self.g]), "broadcast row is not gBest"
+                full.sync(self.losses, t, lam, want_gbest=True)
+                assert np.array_equal(full.gbest, self.pre[self.g])
 
     eng = Engine()
-    drv = sharded.ShardedSync(eng, counts, N, torch.device("cpu"))
+    drv = sharded.ShardedSync(eng, counts, N, torch.device("cpu"), pieces=3, quantum=4)
+    assert drv.bounds == [(0, 88), (88, 176), (176, 257)]
     gs = []
     table = np.array([[5, 4, 3, 2, 1], [1, 2, 3, 4, 5], [2, 2, 1, 1, 3]], np.float32)
     for s in range(3):
         mine = torch.from_numpy(table[s, first:first + counts[r.rank]].copy())
         gs.append(drv.sync(mine))
         assert np.array_equal(eng.losses, table[s]), "all-gather order"
-    print(json.dumps({"rank": r.rank, "g": gs, "copies": eng.log}))
+    print(json.dumps({"rank": r.rank, "g": gs, "log": eng.log}))
     replicas.finish(r)
 """)
 
@@ -132,8 +136,11 @@ def test_sharded_exchange_two_gloo_ranks(tmp_path):
         assert p.returncode == 0, err
     res = [json.loads(o[0].strip().splitlines()[-1]) for o in outs]
     assert res[0]["g"] == res[1]["g"] == [4, 0, 2]
-    # the owner of each gBest (and only it) copied its row out: g=4 -> rank 1 row 1, g=0 -> rank 0 row 0, g=2 -> rank 0 row 2
-    assert res[0]["copies"] == [["copy", 0], ["copy", 2]] and res[1]["copies"] == [["copy", 1]]
+    # every sync updates the three ranges left to right on both ranks; the owner of each gBest
+    # (and only it) hands out its own row: g=4 -> rank 1 row 1, g=0 -> rank 0 row 0, g=2 -> rank 0 row 2
+    ranges = [["range", 0, 88], ["range", 88, 176], ["range", 176, 257]]
+    assert res[0]["log"] == ranges + [["row", 0]] + ranges + [["row", 2]] + ranges
+    assert res[1]["log"] == [["row", 1]] + ranges + ranges + ranges
 
 
 def test_shard_ownership_and_traffic():
@@ -143,3 +150,7 @@ def test_shard_ownership_and_traffic():
     t = sharded.bytes_received_per_sync(11_173_962, [2] * 8)
     assert t["gbest_broadcast"] == 4 * 11_173_962 and t["gather_all_particles"] == 4 * 11_173_962 * 14
     assert t["losses_all_gather"] == 64
+    assert sharded.range_bounds(10, 3, 4) == [(0, 4), (4, 8), (8, 10)]
+    assert sharded.range_bounds(11_173_962, 6) == [(i * 1_862_656, min(11_173_962, (i + 1) * 1_862_656))
+                                                   for i in range(6)]
+    assert sharded.range_bounds(100, 6) == [(0, 100)]

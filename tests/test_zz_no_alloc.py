@@ -74,3 +74,19 @@ def test_static_scratch_unaligned_rows_and_limit():
     assert e.value.code == binding.PSOPS_EINVAL
     torch.cuda.synchronize()
     assert torch.equal(loss, before)
+
+
+def test_static_scratch_exactly_at_its_limit():
+    """K * ceil(N / 128) equal to the size of the built-in array: the last slot
+    is used, the call is accepted and agrees with the workspace route."""
+    gpu_util.ensure_library()
+    K, N = 2, 128 * (binding.PSOPS_STATIC_SCRATCH_DOUBLES // 2)
+    gen = torch.Generator(device="cuda").manual_seed(7)
+    dx = torch.randn((K, N), device="cuda", generator=gen)
+    dd = torch.rand(N, device="cuda", generator=gen) * 1.5 + 0.5
+    dt = torch.randn(N, device="cuda", generator=gen)
+    want = _with_workspace(dx, dd, dt, N)
+    loss = torch.full((K,), -1.0, device="cuda")
+    binding.psops_quadratic_fitness_static(dx, N, K, N, dd, dt, loss)
+    assert np.array_equal(loss.cpu().numpy().view(np.uint32), want.view(np.uint32))
+    assert K * ((N + 127) // 128) == binding.PSOPS_STATIC_SCRATCH_DOUBLES
