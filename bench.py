@@ -324,10 +324,13 @@ def _rel_err(got, want):
     under the parity contract |gpu - ref| <= 1e-6 max(|ref|, 1e-6 RMS(ref))."""
     rms = float(np.sqrt(np.mean(np.square(want, dtype=np.float64)))) if want.size else 0.0
     scale = np.maximum(np.abs(want).astype(np.float64), 1e-6 * rms if rms > 0 else 1e-300)
-    err = np.abs(got.astype(np.float64) - want.astype(np.float64)) / scale
-    same = (got.view(np.uint32) == want.view(np.uint32)) | ((got == 0) & (want == 0))
+    same = (got.view(np.uint32) == want.view(np.uint32)) | ((got == 0) & (want == 0)) \
+        | (np.isnan(got) & np.isnan(want))
+    with np.errstate(invalid="ignore", over="ignore"):
+        err = np.abs(got.astype(np.float64) - want.astype(np.float64)) / scale
     err = np.where(same, 0.0, err)
-    return float(np.nanmax(err)) if err.size else 0.0, int((~(err <= 1e-6)).sum()), int((~same).sum())
+    err = np.where(np.isnan(err), np.inf, err)            # a NaN on one side only is a mismatch
+    return float(err.max()) if err.size else 0.0, int((err > 1e-6).sum()), int((~same).sum())
 
 
 def parity_after_timing(w, sw, made, cols, dtable, dev):
@@ -550,18 +553,20 @@ def run_shards(args, w, dev, dev_index, ranks, peak, peak_src):
             dv[r, :w.N] = torch.from_numpy(workloads.v_row(w, first + r)).to(dev)
     sw = binding.Swarm(dx, dv, dx.clone(), N=w.N, m_max=w.omega, m_min=w.omega, c1=w.c1, c2=w.c2,
                        seed=w.seed, k_first=first, K_total=w.K)
-    drv = sharded.ShardedSync(sharded.swarm_engine(sw), counts, w.N, dev, pieces=args.pieces, timing=True)
+    drv = sharded.ShardedSync(sharded.swarm_engine(sw), counts, w.N, dev, pieces=args.pieces)
     table = torch.from_numpy(workloads.losses(w)).to(dev)
     sampler = ClockSampler(dev_index)
 
     def step(i):
         drv.sync(table[i % table.shape[0], first:first + n_here], 0, w.lam)
 
-    for i in range(args.warmup):
+    timing, made, launches = time_region(step, args.steps, args.warmup, ranks, sampler,
+                                         counter=lambda: sw.launches)
+    # the phases of a sync, from a second short pass with an event between them (the events cost host
+    # time, so they stay out of the timed region above)
+    drv.timing = True
+    for i in range(made, made + 20):
         step(i)
-    drv.timings_ms()                                 # drop the warm-up's events
-    timing, _, launches = time_region(step, args.steps, 0, ranks, sampler, counter=lambda: sw.launches,
-                                      first=args.warmup)
     phases = drv.timings_ms()
     seconds = timing.seconds
     slowest = replicas.max_over_ranks(ranks, seconds)
@@ -721,8 +726,9 @@ def other_rows(args, dev, ranks, peak):
         for name in (() if args.n else ("cfg1", "cfg2")):
             ws = workloads.CONFIGS[name]
             cols = workloads.sample_columns_dense(ws.N, PARITY_COLUMNS, ws.seed) if check else None
-            sw, timing, made, launches, _, dtable = time_sync_workload(ws, dev, 200, 10, ranks, min_seconds=0.05,
-                                                                       cols=cols)
+            # no further windows here: cfg2's omega = 0.9, c = 2 lies outside PSO's stability region, and a
+            # few hundred syncs beyond its 50 would overflow fp32 and leave nothing finite to compare
+            sw, timing, made, launches, _, dtable = time_sync_workload(ws, dev, 200, 10, ranks, cols=cols)
             st = timing.stats(200)
             rows[name + "_sync"] = {"us_per_step": timing.seconds / 200 * 1e6, "value": ws.K * ws.N * 200 / timing.seconds,
                                     "unit": UNIT, "launches_per_sync": launches / 200,

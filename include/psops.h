@@ -144,10 +144,10 @@ int psops_set_losses(psops_ctx *ctx, const float *losses, int on_device);
  * pBest_loss and the counter (no block waits for another).  Otherwise, or with
  * PSOPS_SEPARATE_SELECT, a selection kernel runs first and the update kernel
  * behind it.  The results are identical bit for bit.
- * Cache policy: a swarm whose state (12 bytes per particle-element) is at most
- * three quarters of the GPU's L2 cache is accessed with ordinary loads and
- * stores so that the next sync finds it there; larger swarms are streamed
- * (evict-first).
+ * Cache policy: of the arrays x, v, pbest (4 K N bytes each) as many as fit
+ * together in about half of the GPU's L2 cache are accessed with ordinary
+ * loads and stores, so that the next sync finds them there; the others, and
+ * everything in a swarm far larger than L2, are streamed (evict-first).
  * Errors: EINVAL (t_iter < 0, lambda < 1 or not finite), ESTATE (no losses
  * yet), ECUDA.
  */

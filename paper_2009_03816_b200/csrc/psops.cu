@@ -39,11 +39,19 @@
 #define PSOPS_HOST_CHUNK_BYTES (64ll << 20)
 #endif
 
-// A swarm whose state (12 bytes per particle-element) is at most this share of
-// the L2 cache is accessed with ordinary write-back loads and stores instead
-// of evict-first ones.
+// Share of the L2 cache that the arrays kept resident (write-back accesses
+// instead of evict-first ones) may take up together.  Measured on B200 (126 MB
+// of L2, K = 8, time per sync from a CUDA graph, arrays of 4 K N bytes each):
+//   array   all streamed   x resident   x, v resident   all resident
+//   19 MB      13.6 us        13.3          13.2            13.1
+//   32 MB      24.3           23.1          22.5            24.9
+//   40 MB      33.5           30.5          30.6            34.4
+//   64 MB      52.8           46.5          54.2            53.7
+//   80 MB      66.8           64.5          69.0            67.8
+//  102 MB      82.4           85.0          85.0            83.8
+// i.e. keep as many arrays as fit in about half of L2.
 #ifndef PSOPS_L2_RESIDENT_PERCENT
-#define PSOPS_L2_RESIDENT_PERCENT 75
+#define PSOPS_L2_RESIDENT_PERCENT 52
 #endif
 
 namespace {
@@ -134,7 +142,7 @@ struct psops_ctx {
     int *h_g;                          // page-locked, device-mapped word the selection kernel writes g to (shards)
     int *d_g;                          // the same word as the device sees it
     cudaEvent_t ev_select;             // recorded behind the selection kernel of a shard
-    bool stream_policy;                // true: evict-first accesses (state larger than L2)
+    int resident_arrays;               // how many of x, v, pbest are accessed write-back (kept in L2); the rest is streamed
     long long one_wave_blocks;         // blocks of the select-in-update kernel that are resident at once on this GPU
     int Kt;                            // particles in the whole swarm (= cfg.K unless sharded)
     uint32_t step;                     // syncs enqueued through this context (the stream's own counter is on the device)
@@ -237,28 +245,43 @@ cudaError_t launch_serialized(bool programmatic, void (*kernel)(Params...), dim3
 
 using UpdateKernel = void (*)(const UpdateParams);
 
-// aligned | fitness << 1 | select << 2 | stream << 3  (select and fitness never together)
-UpdateKernel pick_update_kernel(bool aligned, bool fitness, bool select, bool stream)
+// Particles in flight per thread.  With few rows (K <= kFewParticles) a deep
+// batch is mostly empty; one particle at a time needs half the registers, so
+// that five blocks instead of three are resident per SM, which is what a short
+// per-thread loop needs to keep the memory system busy (measured on B200 with
+// 11 M elements: K = 1: 4.1 -> 6.2 TB/s, K = 2: 5.3 -> 6.7, K = 4: 6.3 -> 6.8,
+// K = 8: 6.7 -> 6.8; from K = 16 on the two are equal).  A grid of at most one
+// wave is bound by latency instead, and there the deep batch stays (its loads
+// are all in flight at once): that is also where the selection is folded in.
+constexpr int kFewParticles = 8;
+constexpr int kUnrollFew = 1;
+
+// All instantiations of kernel (b) for one alignment and one cache policy
+// (`resident` arrays of x, v, pbest accessed write-back, the rest streamed).
+struct UpdateKernelSet {
+    UpdateKernel plain, select, few, fitness;
+};
+
+template <bool ALIGNED, int RESIDENT>
+constexpr UpdateKernelSet update_kernel_set()
 {
-    static const UpdateKernel table[16] = {
-        psops_update_kernel<false, false, false, false, kUnroll, kQuads>,
-        psops_update_kernel<true, false, false, false, kUnroll, kQuads>,
-        psops_update_kernel<false, true, false, false, kFitUnroll, kFitQuads>,
-        psops_update_kernel<true, true, false, false, kFitUnroll, kFitQuads>,
-        psops_update_kernel<false, false, true, false, kUnroll, kQuads>,
-        psops_update_kernel<true, false, true, false, kUnroll, kQuads>,
-        nullptr,
-        nullptr,
-        psops_update_kernel<false, false, false, true, kUnroll, kQuads>,
-        psops_update_kernel<true, false, false, true, kUnroll, kQuads>,
-        psops_update_kernel<false, true, false, true, kFitUnroll, kFitQuads>,
-        psops_update_kernel<true, true, false, true, kFitUnroll, kFitQuads>,
-        psops_update_kernel<false, false, true, true, kUnroll, kQuads>,
-        psops_update_kernel<true, false, true, true, kUnroll, kQuads>,
-        nullptr,
-        nullptr,
+    return {psops_update_kernel<ALIGNED, false, false, RESIDENT, kUnroll, kQuads>,
+            psops_update_kernel<ALIGNED, false, true, RESIDENT, kUnroll, kQuads>,
+            psops_update_kernel<ALIGNED, false, false, RESIDENT, kUnrollFew, kQuads>,
+            psops_update_kernel<ALIGNED, true, false, RESIDENT, kFitUnroll, kFitQuads>};
+}
+
+UpdateKernel pick_update_kernel(bool aligned, bool fitness, bool select, int resident, bool few)
+{
+    static const UpdateKernelSet sets[2][4] = {
+        {update_kernel_set<false, 0>(), update_kernel_set<false, 1>(), update_kernel_set<false, 2>(),
+         update_kernel_set<false, 3>()},
+        {update_kernel_set<true, 0>(), update_kernel_set<true, 1>(), update_kernel_set<true, 2>(),
+         update_kernel_set<true, 3>()},
     };
-    return table[(aligned ? 1 : 0) | (fitness ? 2 : 0) | (select ? 4 : 0) | (stream ? 8 : 0)];
+    if (resident < 0 || resident > 3 || (fitness && select)) return nullptr;
+    const UpdateKernelSet &set = sets[aligned ? 1 : 0][resident];
+    return fitness ? set.fitness : select ? set.select : few ? set.few : set.plain;
 }
 
 // One launch of kernel (b) over quads [q_begin, q_end).  `select`: the launch
@@ -286,7 +309,8 @@ int launch_update(psops_ctx *ctx, float m, float k1, float k2, long long q_begin
     const long long span = q_end - q_begin;
     const int per_block = kUpdateThreads * (fitness ? kFitQuads : kQuads);
     const unsigned blocks = (unsigned)((span + per_block - 1) / per_block);
-    const UpdateKernel kernel = pick_update_kernel(ctx->aligned, fitness, select, ctx->stream_policy);
+    const bool few = ctx->cfg.K <= kFewParticles && (long long)blocks > ctx->one_wave_blocks;
+    const UpdateKernel kernel = pick_update_kernel(ctx->aligned, fitness, select, ctx->resident_arrays, few);
     if (kernel == nullptr) return PSOPS_EINVAL;
     const cudaError_t e = launch_serialized(programmatic, kernel, dim3(blocks, 1, 1), dim3(kUpdateThreads, 1, 1), stream, P);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "psops_update_kernel launch");
@@ -410,25 +434,31 @@ int psops_create(psops_ctx **out, const psops_config *cfg, float *d_x, float *d_
 
     int rc = PSOPS_OK;
     cudaError_t e = cudaGetDevice(&ctx->device);
-    // Cache policy of the streaming kernels: evict-first unless the whole state
-    // (x, v, pbest) fits in the device's L2 with room to spare, in which case
-    // the next sync finds it there.
-    ctx->stream_policy = true;
+    // Cache policy of the update kernel: as many of the arrays x, v, pbest as fit
+    // in the given share of the device's L2 are accessed write-back, so that the
+    // next sync finds them there; the rest is streamed (evict-first) past them.
+    ctx->resident_arrays = 0;
     if (e == cudaSuccess) {
         int l2_bytes = 0;
         e = cudaDeviceGetAttribute(&l2_bytes, cudaDevAttrL2CacheSize, ctx->device);
-        const double state_bytes = 12.0 * (double)cfg->K * (double)cfg->N;
-        if (e == cudaSuccess && state_bytes <= (double)l2_bytes * (PSOPS_L2_RESIDENT_PERCENT / 100.0))
-            ctx->stream_policy = false;
+        const double array_bytes = 4.0 * (double)cfg->K * (double)cfg->N;
+        const double room = (double)l2_bytes * (PSOPS_L2_RESIDENT_PERCENT / 100.0);
+        if (e == cudaSuccess) {
+            while (ctx->resident_arrays < 3 && (ctx->resident_arrays + 1) * array_bytes <= room)
+                ctx->resident_arrays += 1;
+#ifdef PSOPS_RESIDENT_FROM_ENV               /* tuning builds only */
+            if (const char *forced = std::getenv("PSOPS_RESIDENT")) ctx->resident_arrays = std::atoi(forced);
+#endif
+        }
     }
     // How many blocks of the single-launch form of a sync run at the same time.
     ctx->one_wave_blocks = 0;
-    if (e == cudaSuccess && cfg->K <= 32) {
+    if (e == cudaSuccess) {
         int sms = 0, per_sm = 0;
         e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device);
         if (e == cudaSuccess)
             e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-                &per_sm, pick_update_kernel(ctx->aligned, false, true, ctx->stream_policy), kUpdateThreads, 0);
+                &per_sm, pick_update_kernel(ctx->aligned, false, true, ctx->resident_arrays, false), kUpdateThreads, 0);
         ctx->one_wave_blocks = (long long)sms * per_sm;
     }
     if (e == cudaSuccess) {

@@ -112,10 +112,11 @@ __device__ __forceinline__ float uniform24(uint32_t w)
 
 // Load / store of one quad.  nvalid = 4 on the vector path means a full
 // 128-bit access; anything else goes element by element under a bound.
-// STREAM: evict-first accesses for a state far larger than L2 (every value is
+// STREAM: evict-first accesses for data far larger than L2 (every value is
 // touched once per sync, so keeping it only displaces the gBest row); with
-// STREAM off the accesses are ordinary write-back ones, for a state that fits
-// in L2 and is found there again by the next sync.
+// STREAM off the accesses are ordinary write-back ones, for data that fits
+// in L2 and is found there again by the next sync.  The update kernel takes
+// the choice per array (x, v, pbest): see its RESIDENT parameter.
 template <bool ALIGNED, bool STREAM = true>
 __device__ __forceinline__ void load_quad(const float *ptr, int nvalid, float (&a)[4])
 {
@@ -347,12 +348,21 @@ psops_select_kernel(const float *loss, float *loss_keep, float *__restrict__ pbe
 // old pBest_loss or step counter, and the block that finishes LAST -- known
 // from a ticket counter, no block ever waits for another -- publishes g, the
 // improved mask, the new pBest_loss and the advanced step counter.
+//
+// RESIDENT = how many of the arrays x, v, pbest (in that order) are accessed
+// with ordinary write-back loads and stores; the rest is streamed evict-first.
+// 0 for a swarm far larger than L2; 3 for one that fits; 1 or 2 in between:
+// the streamed arrays then pass through L2 without displacing the resident
+// ones, which the next sync finds there (x and v are read AND written each
+// sync, pbest only one of the two, hence the order).
 // ---------------------------------------------------------------------------
-template <bool ALIGNED, bool FITNESS, bool SELECT, bool STREAM, int U, int Q>
+template <bool ALIGNED, bool FITNESS, bool SELECT, int RESIDENT, int U, int Q>
 __global__ void PSOPS_UPDATE_BOUNDS
 psops_update_kernel(const __grid_constant__ UpdateParams P)
 {
     static_assert(!(SELECT && FITNESS), "the single-launch form carries no fitness");
+    static_assert(RESIDENT >= 0 && RESIDENT <= 3, "x, v, pbest");
+    constexpr bool STREAM_X = RESIDENT < 1, STREAM_V = RESIDENT < 2, STREAM_P = RESIDENT < 3;
     const long long q0 = P.q_begin + (long long)blockIdx.x * (kUpdateThreads * Q) + threadIdx.x;
     // Whatever follows in the stream with programmatic serialisation (the
     // fitness finaliser, the next sync) may be made resident now; it waits for
@@ -424,7 +434,7 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
 #pragma unroll
     for (int j = 0; j < Q; ++j) {
         load_quad_cached<ALIGNED>(gsrc + col[j], nvalid[j], gb[j]);
-        if (keep_copy) store_quad<ALIGNED, STREAM>(P.gbest_copy + col[j], nvalid[j], gb[j]);
+        if (keep_copy) store_quad<ALIGNED, STREAM_X>(P.gbest_copy + col[j], nvalid[j], gb[j]);
         if (FITNESS) {
             load_quad_cached<ALIGNED>(P.dvec + col[j], nvalid[j], dv[j]);
             load_quad_cached<ALIGNED>(P.tvec + col[j], nvalid[j], tv[j]);
@@ -473,9 +483,9 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
 #pragma unroll
                 for (int j = 0; j < Q; ++j) {
                     const size_t at = row + (size_t)u * (size_t)P.ld + col[j];
-                    load_quad<ALIGNED, STREAM>(P.x + at, nvalid[j], xo[u][j]);
-                    load_quad<ALIGNED, STREAM>(P.v + at, nvalid[j], vo[u][j]);
-                    if (!imp[u]) load_quad<ALIGNED, STREAM>(P.p + at, nvalid[j], pp[u][j]);
+                    load_quad<ALIGNED, STREAM_X>(P.x + at, nvalid[j], xo[u][j]);
+                    load_quad<ALIGNED, STREAM_V>(P.v + at, nvalid[j], vo[u][j]);
+                    if (!imp[u]) load_quad<ALIGNED, STREAM_P>(P.p + at, nvalid[j], pp[u][j]);
                 }
             }
         }
@@ -513,9 +523,9 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
                         vn[e] = __fmaf_rn(t2, dg, __fmaf_rn(t1, dl, a0));  // Eq. 6
                         xn[e] = __fadd_rn(w, vn[e]);                        // Eq. 7
                     }
-                    store_quad<ALIGNED, STREAM>(P.v + at, nvalid[j], vn);
-                    store_quad<ALIGNED, STREAM>(P.x + at, nvalid[j], xn);
-                    if (imp[u]) store_quad<ALIGNED, STREAM>(P.p + at, nvalid[j], xo[u][j]);
+                    store_quad<ALIGNED, STREAM_V>(P.v + at, nvalid[j], vn);
+                    store_quad<ALIGNED, STREAM_X>(P.x + at, nvalid[j], xn);
+                    if (imp[u]) store_quad<ALIGNED, STREAM_P>(P.p + at, nvalid[j], xo[u][j]);
                     if (FITNESS) fq[j][u] = fitness_quad_sum(xn, dv[j], tv[j], nvalid[j]);
                 }
             }

@@ -95,8 +95,13 @@ class ShardedSync:
     def sync(self, local_losses: torch.Tensor, t_iter: int = 0, lam: float = 1.0) -> int:
         """local_losses: this rank's counts[rank] losses (tensor on self.device)."""
         e0 = self._mark()
-        if self.world > 1:
-            # equal-sized pieces (collectives want them): pad to the largest shard
+        if self.world > 1 and len(set(self.counts)) == 1:
+            # equal shards: one collective straight into the K-float buffer
+            dist.all_gather_into_tensor(self.all_losses, local_losses.to(self.device, torch.float32).contiguous(),
+                                        group=self.group)
+            self.engine.set_losses(self.all_losses)
+        elif self.world > 1:
+            # unequal shards: equal-sized pieces (collectives want them), padded to the largest shard
             widest = max(self.counts)
             mine = torch.zeros(widest, dtype=torch.float32, device=self.device)
             mine[:self.counts[self.rank]] = local_losses.to(self.device, torch.float32)
@@ -106,9 +111,9 @@ class ShardedSync:
             for piece, n in zip(pieces, self.counts):
                 self.all_losses[at:at + n] = piece[:n]
                 at += n
+            self.engine.set_losses(self.all_losses)
         else:
-            self.all_losses.copy_(local_losses)
-        self.engine.set_losses(self.all_losses)
+            self.engine.set_losses(local_losses)    # one rank holds the whole swarm: nothing to gather
         g = self.engine.shard_select()              # the same on every rank
         e1 = self._mark()
         owner, row = owner_of(g, self.counts)

@@ -1,78 +1,84 @@
-"""Algorithm 1 end to end on a toy problem: K workers take local gradient steps
-on their own noisy shard of a quadratic objective (plain torch ops stand in for
-local training, which is not part of the library) and synchronise every `step`
-iterations with PSO-PS, with parameter averaging, or -- at step = 1 -- with
-SSGD.  A sanity check that the three synchronisation methods of Section II-B /
-Section III drive the same objective down when called through the library."""
+"""Algorithm 1 end to end on the quadratic stand-in objective (the demo module:
+local gradient steps between synchronisations, PSO-PS / parameter averaging /
+SSGD through the library) with the CPU oracle run beside the library at every
+synchronisation: it is handed the same post-local-step weights and must
+produce the same selection and the same new state."""
+import json
+
 import numpy as np
 import pytest
-import torch
 
-from paper_2009_03816_b200 import binding
+import oracle
+from paper_2009_03816_b200 import demo
 
-import gpu_util
+from gpu_util import NTHREADS, assert_close
 
 pytestmark = pytest.mark.gpu
 
-K, N, STEP, ITERS_PER_EPOCH, EPOCHS, ETA = 8, 50_000, 10, 40, 5, 0.05
+CFG = demo.DemoConfig(K=8, N=20_003, epochs=5, iters_per_epoch=20, step=10, seed=3)
 
 
-def _problem(seed=0):
-    g = torch.Generator(device="cuda").manual_seed(seed)
-    d = torch.rand(N, device="cuda", generator=g) * 1.5 + 0.5
-    t = torch.randn(N, device="cuda", generator=g)
-    shard_t = t + 0.3 * torch.randn((K, N), device="cuda", generator=g)       # each worker's data differs
-    w0 = torch.randn(N, device="cuda", generator=g).repeat(K, 1).contiguous()  # Algorithm 1: same initial weights
-    return d, t, shard_t, w0
+def _problem_on_host(cfg):
+    d, t, shard_t, w0 = demo.problem(cfg, "cuda:0")
+    return d.cpu().numpy(), t.cpu().numpy(), w0.cpu().numpy()
 
 
-def _global_loss(w, d, t):
-    return (d * (w - t) ** 2).sum(dim=1)
+def test_pso_arm_with_the_oracle_in_the_loop():
+    cfg = CFG
+    d, t, w0 = _problem_on_host(cfg)
+    start = np.tile(w0, (cfg.K, 1))
+    ref = oracle.RefSwarm(start, np.zeros_like(start), start, m_max=cfg.m_max, m_min=cfg.m_min,
+                          t_max=cfg.t_max, c1=cfg.c1, c2=cfg.c2, seed=cfg.seed, nthreads=NTHREADS)
+    seen = []
+
+    def observer(ev):
+        # local training happened outside the library and outside the oracle:
+        # the oracle takes the weights as trained, everything else is its own
+        ref.x[:] = ev["x"]
+        loss = oracle.quadratic_losses(ref.x, d, t, nthreads=NTHREADS)
+        assert np.array_equal(loss.view(np.uint32), ev["losses"].view(np.uint32)), ev["iteration"]
+        ref.sync(loss, ev["iteration"], ev["lambda"])
+        assert ev["g"] == ref.g and np.array_equal(ev["improved"], ref.improved), ev["iteration"]
+        assert np.array_equal(ev["pbest_loss"].view(np.uint32), ref.pbest_loss.view(np.uint32))
+        inexact = 0
+        for got, want, name in ((ev["x_after"], ref.x, "x"), (ev["v_after"], ref.v, "v"), (ev["p_after"], ref.p, "pbest")):
+            inexact += assert_close(got, want, f"sync at iteration {ev['iteration']} {name}")
+        assert inexact == 0
+        seen.append(ev["iteration"])
+
+    out = demo.run("pso", cfg, observer=observer)
+    assert seen == list(range(cfg.step, cfg.t_max + 1, cfg.step)) and out["syncs"] == len(seen)
+    assert len(out["best_loss"]) == cfg.epochs
+    assert out["best_loss"][-1] < 0.05 * out["initial_loss"]
 
 
-def _local_grad(w, d, shard_t):
-    return 2.0 * d * (w - shard_t)
+def test_pa_and_ssgd_arms_with_the_oracle_in_the_loop():
+    cfg = CFG
+    checked = {"pa": 0, "ssgd": 0}
+
+    def observer(ev):
+        want = ev["x"].copy()
+        if ev["method"] == "pa":
+            oracle.average(want, nthreads=NTHREADS)
+        else:
+            oracle.ssgd(want, ev["grad"], ev["alpha"], nthreads=NTHREADS)
+        assert np.array_equal(ev["x_after"].view(np.uint32), want.view(np.uint32)), (ev["method"], ev["iteration"])
+        checked[ev["method"]] += 1
+
+    pa = demo.run("pa", cfg, observer=observer)
+    ssgd = demo.run("ssgd", cfg, observer=observer)
+    assert checked == {"pa": cfg.t_max // cfg.step, "ssgd": cfg.t_max}
+    for out in (pa, ssgd):
+        assert out["best_loss"][-1] < 0.05 * out["initial_loss"]
+    # averaging and gradient averaging cancel the shards' pull: they end far below one worker's shard noise
+    shard_floor = cfg.shard_sigma ** 2 * 1.25 * cfg.N
+    assert pa["best_loss"][-1] < 0.5 * shard_floor and ssgd["best_loss"][-1] < 0.5 * shard_floor
 
 
-def _run(method):
-    gpu_util.ensure_library()
-    d, t, shard_t, w0 = _problem()
-    x, v, p = w0.clone(), torch.zeros_like(w0), w0.clone()
-    t_max = EPOCHS * ITERS_PER_EPOCH
-    sw = binding.Swarm(x, v, p, m_max=0.9, m_min=0.3, t_max=t_max, c1=0.2, c2=0.9, seed=11,
-                       flags=binding.PSOPS_QUADRATIC)
-    first = float(_global_loss(x, d, t).min())
-    period = 1 if method == "ssgd" else STEP
-    for it in range(1, t_max + 1):
-        grad = _local_grad(x, d, shard_t)
-        if method == "ssgd":
-            sw.ssgd(grad, -ETA)                                   # w <- w + (alpha / n) sum grad_k, alpha = -eta
-            continue
-        x -= ETA * grad                                           # Algorithm 1: "update w by SGD"
-        if it % period == 0:
-            if method == "pa":
-                sw.average()
-            else:
-                sw.set_quadratic(d, t)
-                sw.eval_quadratic()                               # fitness = loss of the current weights
-                binding.psops_set_quadratic(sw.ctx, None, None)   # detach: the losses of the weights as
-                sw.sync(it, 1.0 + (it - 1) // ITERS_PER_EPOCH)    # trained are wanted, not those after the sync
-    torch.cuda.synchronize()
-    last = float(_global_loss(x, d, t).min())
-    spread = float((x - x.mean(dim=0)).abs().max())
-    sw.close()
-    return first, last, spread
-
-
-def test_three_synchronisation_methods_reduce_the_objective():
-    res = {m: _run(m) for m in ("pso", "pa", "ssgd")}
-    noise_floor = 0.3 ** 2 * 1.25 * N            # a worker that fits only its own shard ends near here
-    for m, (first, last, spread) in res.items():
-        assert last < 0.05 * first, (m, first, last)
-        assert np.isfinite(last)
-    # averaging and gradient averaging cancel most of the shard noise; PSO-PS keeps
-    # the workers apart (it is a search, not a consensus) but must not be worse than
-    # a worker left alone with its shard
-    assert res["pa"][1] < 0.5 * noise_floor and res["ssgd"][1] < 0.5 * noise_floor
-    assert res["pso"][1] < 1.5 * noise_floor
-    assert res["ssgd"][2] == 0.0                 # SSGD hands every worker the same weights
+def test_demo_main_prints_three_curves(capsys):
+    out = demo.main(["--epochs", "3", "--iters-per-epoch", "10", "--n", "4099", "--k", "4"])
+    printed = json.loads(capsys.readouterr().out.strip().splitlines()[-1])
+    assert printed == out and set(out["methods"]) == {"pso", "pa", "ssgd"}
+    for m in out["methods"].values():
+        assert len(m["best_loss"]) == 3 and all(np.isfinite(m["best_loss"]))
+        assert m["best_loss"][-1] < m["initial_loss"]

@@ -114,6 +114,13 @@ SHARD_WORKER = textwrap.dedent("""
         mine = torch.from_numpy(table[s, first:first + counts[r.rank]].copy())
         gs.append(drv.sync(mine))
         assert np.array_equal(eng.losses, table[s]), "all-gather order"
+    # equal shards take the single-collective gather: same losses in the same order
+    class Probe(Engine):
+        def shard_update_range(self, gbest, a, b, t, lam): pass
+    probe = Probe()
+    drv2 = sharded.ShardedSync(probe, [2, 2], N, torch.device("cpu"), pieces=1)
+    drv2.sync(torch.tensor([10.0 + r.rank, 20.0 + r.rank]))
+    assert probe.losses.tolist() == [10.0, 20.0, 11.0, 21.0], probe.losses
     print(json.dumps({"rank": r.rank, "g": gs, "log": eng.log}))
     replicas.finish(r)
 """)
