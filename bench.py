@@ -36,13 +36,15 @@ METRIC = "pso_sync_throughput"
 UNIT = "particle-elements/s"
 FALLBACK_HBM_GBS = 6650.0           # earlier measurement on this machine, used only if no measured file
 
-# DRAM traffic of the fused update kernel from an ncu capture, per
-# particle-element, and the hash of the source it was taken from: everything in
-# psops_kernels.cuh up to the averaging kernel, i.e. the update kernel and all
-# it uses.  The benchmark reports null once that text has changed.
-NCU_TRAFFIC = {"source_sha256": "ada5eebaa22a962d5e61660f02521acb7dc8cc903445cbd8c4328c8b43ec14c5",
-               "bytes_per_particle_element": 19.93,       # 16.30 GB / 817.8 M: full-size cfg4 launches, 1-pass counters
-               "profile": "profiles/update_kernel_cfg4_n4m_full.txt"}
+# DRAM traffic of the fused update kernel from an ncu capture of a small case
+# (N = 4 M, state larger than L2), per particle-element -- every value is
+# touched once, so traffic grows in proportion to K x N -- and the hash of the
+# source it was taken from: everything in psops_kernels.cuh up to the averaging
+# kernel, i.e. the update kernel and all it uses.  The benchmark reports null
+# once that text has changed, and for workloads whose state is kept in L2.
+NCU_TRAFFIC = {"source_sha256": "d3ccfc37a5e3f180540dfa794a7cc571c95eba65911edc1d9be1d9266547ec8a",
+               "bytes_per_particle_element": 19.57,       # 2.506 / 2.503 GB per launch over 128 M: cfg4 recipe at N = 4 M
+               "profile": "profiles/update_kernel_cfg4_n4m.txt"}
 KERNEL_SOURCE = os.path.join(ROOT, "paper_2009_03816_b200", "csrc", "psops_kernels.cuh")
 HASH_UNTIL = "// Kernel (c): parameter averaging"
 
@@ -600,6 +602,8 @@ def run_shards(args, w, dev, dev_index, ranks, peak, peak_src):
 def ncu_traffic(w):
     if not NCU_TRAFFIC["source_sha256"] or update_kernel_source_sha256() != NCU_TRAFFIC["source_sha256"]:
         return None
+    if 4 * w.K * w.N <= 0.52 * (126 << 20):       # an array is kept in L2: DRAM traffic is not proportional
+        return None
     return NCU_TRAFFIC["bytes_per_particle_element"] * w.K * w.N
 
 
@@ -651,7 +655,7 @@ def _row(w, timing, steps, nbytes, peak, K_here=None, parity=None):
     return out
 
 
-def time_variant(w, dev, ranks, peak, flags=0, shard=None, steps=100):
+def time_variant(w, dev, ranks, peak, flags=0, shard=None, steps=100, min_seconds=0.05):
     """psops_sync with a flag set, or the select + update pair of one particle shard."""
     import torch
     from paper_2009_03816_b200 import binding, workloads
@@ -674,7 +678,7 @@ def time_variant(w, dev, ranks, peak, flags=0, shard=None, steps=100):
             sw.set_losses(table[i % table.shape[0]])
             sw.shard_select()
             sw.shard_update(gbest, 0, w.lam)
-    timing, _, _ = time_region(step, steps, 5, ranks, per_step=True, min_seconds=0.05)
+    timing, _, _ = time_region(step, steps, 5, ranks, per_step=True, min_seconds=min_seconds)
     out = _row(w, timing, steps, 20 * K_here * w.N + 4 * w.N, peak, K_here)
     sw.close()
     del sw
@@ -695,7 +699,7 @@ def other_rows(args, dev, ranks, peak):
         S3, S5, W = args.row_steps or 100, args.row_steps or 50, (5 if not args.row_steps else 3)
         cols = workloads.sample_columns_dense(w3.N, PARITY_COLUMNS, w3.seed) if check else None
         sw, timing, made, _, _, dtable = time_sync_workload(w3, dev, S3, W, ranks, per_step=True,
-                                                            min_seconds=0.1, cols=cols)
+                                                            min_seconds=0.0 if args.row_steps else 0.1, cols=cols)
         par = parity_after_timing(w3, sw, made, cols, dtable, dev) if check else None
         rows["cfg3_sync"] = _row(w3, timing, S3, sync_bytes(w3), peak, parity=par)
         timing, _, _ = time_region(lambda i: sw.average(), S3, W, ranks, per_step=True)
@@ -710,10 +714,11 @@ def other_rows(args, dev, ranks, peak):
         sw.close()
         del sw
         torch.cuda.empty_cache()
-        rows["cfg3_sync_gbest_history"] = time_variant(w3, dev, ranks, peak, flags=4, steps=S3)
+        short = 0.0 if args.row_steps else 0.05          # profiling captures want few launches
+        rows["cfg3_sync_gbest_history"] = time_variant(w3, dev, ranks, peak, flags=4, steps=S3, min_seconds=short)
         # what one GPU of an 8-GPU particle-sharded run does per sync: 2 of the 16 particles,
         # gBest read from a broadcast buffer (the collectives themselves need more than one GPU)
-        rows["cfg3_shard_2_of_16"] = time_variant(w3, dev, ranks, peak, shard=(0, 2), steps=S3)
+        rows["cfg3_shard_2_of_16"] = time_variant(w3, dev, ranks, peak, shard=(0, 2), steps=S3, min_seconds=short)
         sw, timing, _, _, keep, _ = time_sync_workload(w5, dev, S5, W, ranks, fused_fitness=True, per_step=True)
         par = parity_fused_fitness(w5, sw, keep, dev) if check else None
         rows["cfg5_sync_fused_fitness"] = _row(w5, timing, S5, sync_bytes(w5, True), peak, parity=par)

