@@ -316,7 +316,9 @@ int psops_eval_quadratic(psops_ctx *ctx);
  * between calls (every slot that is read has been written by the same call);
  * calls that overlap in time on one GPU overwrite each other's partial results,
  * so keep them on one stream or order them yourself.
- * Errors: EINVAL, EALIGN (a pointer not 4-byte aligned), ELIMIT, ECUDA.
+ * Errors: EINVAL (also: a buffer that is host memory, or device memory of a GPU
+ * other than the current one), EALIGN (a pointer not 4-byte aligned), ELIMIT,
+ * ECUDA.
  */
 #define PSOPS_STATIC_SCRATCH_DOUBLES (1 << 20)
 int psops_quadratic_fitness_static(const float *d_x, int64_t ld, int32_t K, int64_t N,

@@ -1034,6 +1034,22 @@ extern "C" int psops_quadratic_fitness_static(const float *d_x, int64_t ld, int3
     const long long tiles = (N + kTileElems - 1) / kTileElems;
     if ((long long)K * tiles > (long long)PSOPS_STATIC_SCRATCH_DOUBLES) return PSOPS_ELIMIT;
 
+    // The built-in array that is used is the current device's: the buffers must
+    // live there too (a pointer the runtime does not know, e.g. one from another
+    // allocator it cannot see, is let through).
+    int current = -1;
+    if (cudaGetDevice(&current) != cudaSuccess) return PSOPS_ECUDA;
+    const void *buffers[4] = {d_x, d_dvec, d_tvec, d_loss};
+    for (const void *ptr : buffers) {
+        cudaPointerAttributes where{};
+        if (cudaPointerGetAttributes(&where, ptr) != cudaSuccess) {
+            (void)cudaGetLastError();
+            continue;
+        }
+        if (where.type == cudaMemoryTypeHost) return PSOPS_EINVAL;
+        if (where.type == cudaMemoryTypeDevice && where.device != current) return PSOPS_EINVAL;
+    }
+
     double *tile_sums = nullptr;
     const int rc = static_scratch_for_current_device(&tile_sums);
     if (rc != PSOPS_OK) return rc;

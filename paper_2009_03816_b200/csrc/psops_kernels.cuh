@@ -722,7 +722,20 @@ psops_fitness_finalize_kernel(const double *__restrict__ partials, float *__rest
 #pragma unroll
         for (int d = 0; d < D; ++d) acc = __dadd_rn(acc, v[d]);
     }
-    for (; m < tiles; m += kFinalizeThreads) acc = __dadd_rn(acc, row[m]);
+    {
+        // The last, partial batch the same way -- loads first, then the chain of
+        // additions -- so that it costs one memory latency and not one per tile.
+        double v[D];
+#pragma unroll
+        for (int d = 0; d < D; ++d) {
+            v[d] = 0.0;
+            if (m + (long long)d * kFinalizeThreads < tiles)
+                asm volatile("ld.global.f64 %0, [%1];" : "=d"(v[d]) : "l"(row + m + (long long)d * kFinalizeThreads));
+        }
+#pragma unroll
+        for (int d = 0; d < D; ++d)
+            if (m + (long long)d * kFinalizeThreads < tiles) acc = __dadd_rn(acc, v[d]);
+    }
 
 #pragma unroll
     for (int off = 16; off >= 1; off >>= 1)
