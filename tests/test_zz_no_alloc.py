@@ -75,10 +75,7 @@ def test_static_scratch_unaligned_rows_and_limit():
     # a host buffer where a device buffer belongs is refused before anything is launched
     pinned = torch.zeros(K).pin_memory()
     with pytest.raises(binding.PsopsError) as e:
-        load = binding.load()
-        rc = load.psops_quadratic_fitness_static(dx.data_ptr(), 1001, K, N, dd.data_ptr(), dt.data_ptr(),
-                                                 pinned.data_ptr(), None)
-        raise binding.PsopsError(rc, "psops_quadratic_fitness_static") if rc else AssertionError("accepted")
+        binding.psops_quadratic_fitness_static(dx, 1001, K, N, dd, dt, pinned)
     assert e.value.code == binding.PSOPS_EINVAL
     torch.cuda.synchronize()
     assert torch.equal(loss, before)
