@@ -172,3 +172,32 @@ def test_sample_columns_cover_head_and_tail():
     cols = workloads.sample_columns(1000, 50, 3)
     assert cols[0] == 0 and cols[-1] == 999 and np.all(np.diff(cols) > 0)
     assert {0, 1, 2, 3, 996, 997, 998, 999} <= set(cols.tolist())
+
+
+def test_bench_parity_metric_and_timing_stats():
+    """The benchmark's own checker: the error measure of its `parity` object and
+    the per-step statistics (host arithmetic only)."""
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("bench", os.path.join(ROOT, "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    want = np.array([[1.0, 2.0, 0.0, np.nan, np.inf, 4.0]], np.float32)
+    got = want.copy()
+    got[0, 2] = -0.0                                   # +0 / -0 and NaN / NaN count as identical
+    assert bench._rel_err(got, want) == (0.0, 0, 0)
+    got[0, 1] = np.nextafter(np.float32(2.0), np.float32(3.0))      # one ulp: inside 1e-6, not identical
+    err, outside, inexact = bench._rel_err(got, want)
+    assert 0 < err < 1e-6 and outside == 0 and inexact == 1
+    got[0, 5] = 4.001
+    got[0, 0] = np.nan                                 # a NaN on one side only is a mismatch
+    err, outside, inexact = bench._rel_err(got, want)
+    assert err == np.inf and outside == 2 and inexact == 3
+    t = bench.Timing(0.010, [1.0, 3.0, 2.0, 4.0])
+    t.window_ms_per_step = [2.0, 3.0]
+    st = t.stats(4)
+    assert st["ms_per_step_mean"] == 2.5 and st["per_step_ms"] == {"median": 2.5, "min": 1.0, "max": 4.0, "n": 4}
+    assert st["window_ms_per_step"] == {"median": 2.5, "min": 2.0, "max": 3.0, "n": 3}
+    # algorithmic bytes of a sync: 20 B per particle-element + the gBest row
+    from paper_2009_03816_b200 import workloads
+    w = workloads.CONFIGS["cfg4"]
+    assert bench.sync_bytes(w) == 20 * 32 * 25_557_032 + 4 * 25_557_032 == 16_458_728_608
