@@ -162,6 +162,16 @@ def test_cfg2_full():
     assert _run_workload(workloads.CONFIGS["cfg2"], every=7) == 0
 
 
+@pytest.mark.parametrize("N", [500_003, 900_001, 1_600_002, 2_700_001])
+def test_cfg2_recipe_across_the_cache_policies(N):
+    """The update kernel keeps as many of the arrays x, v, pbest in L2 as fit in
+    about half of it and streams the rest: with K = 8 these lengths give arrays
+    of 16, 29, 51 and 86 MB, i.e. all three, two, one and none kept (on a GPU
+    with 126 MB of L2).  The results must not depend on the choice."""
+    w = workloads.CONFIGS["cfg2"].scaled(N=N, S=6)
+    assert _run_workload(w, every=2) == 0
+
+
 def test_cfg3_scaled_with_ties():
     w = workloads.CONFIGS["cfg3"].scaled(N=300_002)
     assert w.N % 4 == 2 and w.ld == 300_032          # ragged last quad, padded pitch
