@@ -91,6 +91,18 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
+def workload_config(w, replicas_count):
+    """The `config` object of the JSON line: names the workload; the same for
+    the GPU arm and for the reference arm (whose bounded sample is described in
+    its `cpu_baseline.sample`)."""
+    return {"workload": f"{w.name}: K={w.K} particles x N={w.N} fp32 ({w.note}), "
+                        f"omega={w.omega}, c1={w.c1}, c2={w.c2}, lambda={w.lam}, seed={w.seed}",
+            "K": w.K, "N": w.N, "ld": w.ld, "replicas": replicas_count,
+            "l2": "state (12*K*N bytes) exceeds L2; no flush needed" if 12 * w.K * w.N > (126 << 20)
+                  else "state fits L2: an L2-resident result, reported as such",
+            "parallelism": "replicas only"}
+
+
 def sync_bytes(w, fused_fitness=False) -> int:
     """Algorithmic bytes of one sync: w, v read and written, pBest read or
     written (20 B per particle-element) plus one read of the gBest row."""
@@ -492,12 +504,7 @@ def run_psops(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{w.name}: K={w.K} particles x N={w.N} fp32 ({w.note}), "
-                               f"omega={w.omega}, c1={w.c1}, c2={w.c2}, lambda={w.lam}, seed={w.seed}",
-                   "K": w.K, "N": w.N, "ld": w.ld, "replicas": ranks.world,
-                   "l2": "state (12*K*N bytes) exceeds L2; no flush needed" if 12 * pe > (126 << 20)
-                         else "state fits L2: an L2-resident result, reported as such",
-                   "parallelism": "replicas only"},
+        "config": workload_config(w, ranks.world),
         "timing": timing.stats(args.steps),
         "clocks": sampler.report(),
         "e2e": e2e,
@@ -836,9 +843,7 @@ def run_reference(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3 / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
-        "config": {"workload": f"{w.name}: K={w.K} particles x N={w.N} fp32 ({w.note}), "
-                               f"omega={w.omega}, c1={w.c1}, c2={w.c2}, lambda={w.lam}, seed={w.seed}",
-                   "K": w.K, "N": w.N, "sample_columns": n_cols},
+        "config": workload_config(w, args.gpus),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": nthreads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,

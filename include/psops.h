@@ -210,8 +210,8 @@ int psops_host_unregister(void *host_ptr);
  * sharded context (they need the whole swarm).  The quadratic fitness and
  * PSOPS_GBEST_HISTORY are not available on shards; PSOPS_KEEP_GBEST is (the
  * shard keeps a copy of the row it was given).
- * Errors: EINVAL, EALIGN, ESTATE (no losses / update without select / a range
- * out of order), ECUDA.
+ * Errors: EINVAL, EALIGN, ESTATE (no losses / update without select / a second
+ * select before the update is complete / a range out of order), ECUDA.
  */
 int psops_shard_select(psops_ctx *ctx, int *g);
 int psops_shard_update(psops_ctx *ctx, int64_t t_iter, float lambda, const float *d_gbest_row);

@@ -637,7 +637,7 @@ int psops_shard_select(psops_ctx *ctx, int *g)
     DeviceGuard device_guard(ctx);
     if (ctx == nullptr || g == nullptr) return PSOPS_EINVAL;
     if (!ctx->have_losses) return PSOPS_ESTATE;
-    if (ctx->selected && ctx->range_next != 0) return PSOPS_ESTATE;     // an update is half done
+    if (ctx->selected) return PSOPS_ESTATE;     // the update of the previous selection is still due (or half done)
     if (ctx->h_g == nullptr) {
         // One word of page-locked host memory that the selection kernel writes
         // directly: the host then needs no copy and no drain of the stream, only

@@ -194,6 +194,9 @@ def test_shards_update_in_ranges_owner_reads_its_own_row_and_gbest_is_kept():
     # ranges must come left to right, on quad boundaries, after a selection
     sw.set_losses(dl)
     sw.shard_select()
+    with pytest.raises(binding.PsopsError) as e:
+        sw.shard_select()                                # a selection whose update is still due
+    assert e.value.code == binding.PSOPS_ESTATE
     for a, b, code in ((4, 8, binding.PSOPS_ESTATE), (0, 6, binding.PSOPS_EINVAL), (0, N + 1, binding.PSOPS_EINVAL)):
         with pytest.raises(binding.PsopsError) as e:
             sw.shard_update_range(received, a, b)
