@@ -136,10 +136,10 @@ int psops_set_losses(psops_ctx *ctx, const float *losses, int on_device);
  * psops_sync recorded into a CUDA graph (with the losses in a device buffer,
  * see psops_set_losses) keeps walking the random stream when the graph is
  * replayed; t_iter and lambda are then the ones given at capture.
- * Launches: a small swarm -- at most 32 particles, no history variant, no fused
+ * Launches: a small swarm -- at most 16 particles, no history variant, no fused
  * fitness, and few enough elements that all thread blocks of the update are
- * resident at once (about 450,000 on a B200) -- is launch-bound, and its whole
- * sync is ONE kernel: every thread block recomputes steps 1 and 2 from the K
+ * resident at once (on a B200 about 450,000 with up to 4 particles, 150,000
+ * with 5 to 16) -- is launch-bound, and its whole sync is ONE kernel: every thread block recomputes steps 1 and 2 from the K
  * losses, and the block that finishes last publishes g, the improved mask,
  * pBest_loss and the counter (no block waits for another).  Otherwise, or with
  * PSOPS_SEPARATE_SELECT, a selection kernel runs first and the update kernel

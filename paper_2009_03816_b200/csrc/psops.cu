@@ -255,11 +255,22 @@ using UpdateKernel = void (*)(const UpdateParams);
 // are all in flight at once): that is also where the selection is folded in.
 constexpr int kFewParticles = 8;
 constexpr int kUnrollFew = 1;
+// The single-launch form (selection folded in) is for launch-bound swarms: at
+// most kSelectMaxParticles particles on a grid of at most one wave.  There the
+// per-thread loop over particles is a chain of memory latencies, so the batch
+// is as deep as the swarm: four particles in flight up to K = 4, eight beyond
+// (152 registers, one block per SM, hence a smaller "one wave").  Measured per
+// sync from a CUDA graph, N = 61,706: K = 4: 4.4 us; K = 8: 6.8 us (7.9 with
+// four in flight, 7.6 as two kernels); K = 16: 12.3 (13.7 / 12.2); K = 32 is
+// faster as two kernels (21 vs 23 us) and keeps them.
+constexpr int kSelectMaxParticles = 16;
+constexpr int kUnrollSelectDeep = 8;
+static_assert(32 % kUnrollSelectDeep == 0 && kSelectMaxParticles <= 32, "one improved-mask word, reloaded every 32 particles");
 
 // All instantiations of kernel (b) for one alignment and one cache policy
 // (`resident` arrays of x, v, pbest accessed write-back, the rest streamed).
 struct UpdateKernelSet {
-    UpdateKernel plain, select, few, fitness;
+    UpdateKernel plain, select, select_deep, few, fitness;
 };
 
 template <bool ALIGNED, int RESIDENT>
@@ -267,11 +278,12 @@ constexpr UpdateKernelSet update_kernel_set()
 {
     return {psops_update_kernel<ALIGNED, false, false, RESIDENT, kUnroll, kQuads>,
             psops_update_kernel<ALIGNED, false, true, RESIDENT, kUnroll, kQuads>,
+            psops_update_kernel<ALIGNED, false, true, RESIDENT, kUnrollSelectDeep, kQuads>,
             psops_update_kernel<ALIGNED, false, false, RESIDENT, kUnrollFew, kQuads>,
             psops_update_kernel<ALIGNED, true, false, RESIDENT, kFitUnroll, kFitQuads>};
 }
 
-UpdateKernel pick_update_kernel(bool aligned, bool fitness, bool select, int resident, bool few)
+UpdateKernel pick_update_kernel(bool aligned, bool fitness, bool select, int resident, bool few, int K)
 {
     static const UpdateKernelSet sets[2][4] = {
         {update_kernel_set<false, 0>(), update_kernel_set<false, 1>(), update_kernel_set<false, 2>(),
@@ -281,7 +293,9 @@ UpdateKernel pick_update_kernel(bool aligned, bool fitness, bool select, int res
     };
     if (resident < 0 || resident > 3 || (fitness && select)) return nullptr;
     const UpdateKernelSet &set = sets[aligned ? 1 : 0][resident];
-    return fitness ? set.fitness : select ? set.select : few ? set.few : set.plain;
+    if (fitness) return set.fitness;
+    if (select) return K > kUnroll ? set.select_deep : set.select;
+    return few ? set.few : set.plain;
 }
 
 // One launch of kernel (b) over quads [q_begin, q_end).  `select`: the launch
@@ -310,7 +324,7 @@ int launch_update(psops_ctx *ctx, float m, float k1, float k2, long long q_begin
     const int per_block = kUpdateThreads * (fitness ? kFitQuads : kQuads);
     const unsigned blocks = (unsigned)((span + per_block - 1) / per_block);
     const bool few = ctx->cfg.K <= kFewParticles && (long long)blocks > ctx->one_wave_blocks;
-    const UpdateKernel kernel = pick_update_kernel(ctx->aligned, fitness, select, ctx->resident_arrays, few);
+    const UpdateKernel kernel = pick_update_kernel(ctx->aligned, fitness, select, ctx->resident_arrays, few, ctx->cfg.K);
     if (kernel == nullptr) return PSOPS_EINVAL;
     const cudaError_t e = launch_serialized(programmatic, kernel, dim3(blocks, 1, 1), dim3(kUpdateThreads, 1, 1), stream, P);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "psops_update_kernel launch");
@@ -458,7 +472,8 @@ int psops_create(psops_ctx **out, const psops_config *cfg, float *d_x, float *d_
         e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device);
         if (e == cudaSuccess)
             e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-                &per_sm, pick_update_kernel(ctx->aligned, false, true, ctx->resident_arrays, false), kUpdateThreads, 0);
+                &per_sm, pick_update_kernel(ctx->aligned, false, true, ctx->resident_arrays, false, cfg->K),
+                kUpdateThreads, 0);
         ctx->one_wave_blocks = (long long)sms * per_sm;
     }
     if (e == cudaSuccess) {
@@ -510,13 +525,14 @@ int psops_sync(psops_ctx *ctx, int64_t t_iter, float lambda)
     const float k2 = ctx->cfg.c2 / lambda;
     const bool fitness = ctx->dvec != nullptr;
 
-    // A small swarm (at most 32 particles, all blocks of the update resident at
+    // A small swarm (at most 16 particles, all blocks of the update resident at
     // once) is launch-bound: there the update launch does the selection itself,
     // one kernel per sync.  Anything larger, the history variant and the fused
     // fitness run the selection kernel first and the update behind it, which
     // costs a large grid nothing and keeps its blocks free of the closing step.
     const long long update_blocks = (ctx->quads + (long long)kUpdateThreads * kQuads - 1) / ((long long)kUpdateThreads * kQuads);
-    const bool select_in_update = ctx->cfg.K <= 32 && !fitness && update_blocks <= ctx->one_wave_blocks &&
+    const bool select_in_update = ctx->cfg.K <= kSelectMaxParticles && !fitness &&
+                                  update_blocks <= ctx->one_wave_blocks &&
                                   !(ctx->cfg.flags & (PSOPS_GBEST_HISTORY | PSOPS_SEPARATE_SELECT));
     if (!select_in_update) {
         rc = launch_select(ctx);

@@ -341,13 +341,15 @@ psops_select_kernel(const float *loss, float *loss_keep, float *__restrict__ pbe
 // contiguous piece of each row, which is what DRAM and the TLB like when K
 // rows x 3 arrays are all being walked at once.
 //
-// SELECT (K <= 32, whole-range launches only): the launch does the selection
+// SELECT (K <= 32 by construction, used up to 16; whole-range launches only): the launch does the selection
 // as well, so that a sync is ONE kernel.  Every warp recomputes Algorithm 3
 // and the pBest comparisons from the K losses (K L2-served floats and a
-// five-stage shuffle), nothing is written while any block may still read the
-// old pBest_loss or step counter, and the block that finishes LAST -- known
-// from a ticket counter, no block ever waits for another -- publishes g, the
-// improved mask, the new pBest_loss and the advanced step counter.
+// five-stage shuffle) and then draws a ticket from an atomic counter.  The
+// block that draws the LAST ticket knows that every block has read the old
+// pBest_loss and step counter -- nobody reads them again in this launch -- and
+// it alone publishes g, the improved mask, the new pBest_loss and the advanced
+// step counter, while its own row loads are in flight.  No block ever waits
+// for another.
 //
 // RESIDENT = how many of the arrays x, v, pbest (in that order) are accessed
 // with ordinary write-back loads and stores; the rest is streamed evict-first.
@@ -373,7 +375,7 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
     // no-op for an ordinary launch).
     asm volatile("griddepcontrol.wait;" ::: "memory");
     if (!FITNESS && !SELECT && q0 >= P.q_end) return;   // with FITNESS whole warps stay for the shuffles,
-                                                        // with SELECT whole blocks for the closing barrier
+                                                        // with SELECT whole blocks for the barrier below
 
     bool active[Q];
     int nvalid[Q];
@@ -408,6 +410,10 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
         c.idx = live ? lane : 0x7fffffff;
         g = warp_best_candidate(c).idx;
         step = __ldcg(&P.desc_pub->next_step);
+        // g and the ballot needed every lane's loads: past this barrier all warps
+        // of the block hold the old selection state in registers, and the block's
+        // ticket (drawn below, under the first row loads) may say so.
+        __syncthreads();
     } else {
         step = P.desc->step;
         g = P.desc->g;
@@ -489,6 +495,28 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
                 }
             }
         }
+        if (SELECT && i0 == 0 && threadIdx.x < 32) {
+            // The ticket, in the shadow of the loads just issued.  Whoever draws the
+            // last one publishes; the others carry on at once.
+            unsigned int ticket = 0;
+            if (lane == 0) ticket = atomicAdd(&P.desc_pub->done, 1u);
+            ticket = __shfl_sync(0xffffffffu, ticket, 0);
+            if (ticket == gridDim.x - 1) {
+                if (lane < P.K) {
+                    P.loss_keep[lane] = sel_loss;                 // the context's own copy of the losses
+                    if (sel_improved) P.pbest_loss[lane] = sel_loss;
+                }
+                if (lane == 0) {
+                    SyncDesc *d = P.desc_pub;
+                    d->g = g;
+                    d->improved[0] = sel_word;
+                    d->from_kept = 0;
+                    d->step = step;
+                    d->next_step = step + 1u;
+                    d->done = 0u;                                 // every ticket of this launch has been drawn
+                }
+            }
+        }
         if (FITNESS) {
             if (fq_i0 >= 0) flush_fitness();     // previous batch, under this batch's loads
 #pragma unroll
@@ -534,37 +562,6 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
     }
     if (FITNESS && fq_i0 >= 0) flush_fitness();
 
-    if (SELECT) {
-        // Every warp of this block read the old selection state before this
-        // barrier; the ticket is taken after it.  The block that draws the last
-        // ticket therefore knows that no block will read that state again, and
-        // it alone moves it on.  Nobody waits: a block that is not last leaves.
-        __syncthreads();
-        if (threadIdx.x < 32) {
-            unsigned int ticket = 0;
-            if (lane == 0) {
-                __threadfence();
-                ticket = atomicAdd(&P.desc_pub->done, 1u);
-            }
-            ticket = __shfl_sync(0xffffffffu, ticket, 0);
-            if (ticket == gridDim.x - 1) {
-                __threadfence();
-                if (lane < P.K) {
-                    P.loss_keep[lane] = sel_loss;                 // the context's own copy of the losses
-                    if (sel_improved) P.pbest_loss[lane] = sel_loss;
-                }
-                if (lane == 0) {
-                    SyncDesc *d = P.desc_pub;
-                    d->g = g;
-                    d->improved[0] = sel_word;
-                    d->from_kept = 0;
-                    d->step = step;
-                    d->next_step = step + 1u;
-                    d->done = 0u;
-                }
-            }
-        }
-    }
 }
 
 // ---------------------------------------------------------------------------

@@ -31,10 +31,11 @@ def _swarm(K, N, seed, sv=0.1):
 # Small shapes: several tiles, ragged tails, both kernels variants.
 # ---------------------------------------------------------------------------
 @pytest.mark.parametrize("N", [1, 2, 3, 5, 127, 128, 129, 1000, 4099])
-@pytest.mark.parametrize("K,separate", [(1, False), (2, False), (3, False), (32, False), (1, True), (2, True),
-                                        (3, True), (32, True), (33, True)])
+@pytest.mark.parametrize("K,separate", [(1, False), (2, False), (3, False), (5, False), (8, False), (16, False),
+                                        (1, True), (2, True), (3, True), (8, True), (32, True), (33, True)])
 def test_small_shapes_vector_path(K, N, separate):
-    """Up to 32 particles a small sync is one launch that selects and updates;
+    """Up to 16 particles a small sync is one launch that selects and updates
+    (four particles in flight up to K = 4, eight beyond);
     PSOPS_SEPARATE_SELECT (and any larger swarm) runs the selection kernel
     first.  Both must follow the oracle bit for bit."""
     x, v, p = _swarm(K, N, 100 * K + N)
@@ -84,7 +85,7 @@ def test_many_particles():
 # ---------------------------------------------------------------------------
 # Selection edge cases through the device kernel.
 # ---------------------------------------------------------------------------
-@pytest.mark.parametrize("K", [20, 32, 40])          # selection inside the update launch / selection kernel
+@pytest.mark.parametrize("K", [7, 12, 16, 20, 40])    # selection inside the update launch (K <= 16) / selection kernel
 def test_selection_ties_nan_inf_on_device(K):
     N = 64
     x, v, p = _swarm(K, N, 9)
