@@ -136,14 +136,20 @@ int psops_set_losses(psops_ctx *ctx, const float *losses, int on_device);
  * psops_sync recorded into a CUDA graph (with the losses in a device buffer,
  * see psops_set_losses) keeps walking the random stream when the graph is
  * replayed; t_iter and lambda are then the ones given at capture.
- * Launches: a small swarm -- at most 16 particles, no history variant, no fused
+ * Launches: a small swarm -- at most 8 particles, no history variant, no fused
  * fitness, and few enough elements that all thread blocks of the update are
  * resident at once (on a B200 about 450,000 with up to 4 particles, 150,000
- * with 5 to 16) -- is launch-bound, and its whole sync is ONE kernel: every thread block recomputes steps 1 and 2 from the K
- * losses, and the block that finishes last publishes g, the improved mask,
- * pBest_loss and the counter (no block waits for another).  Otherwise, or with
+ * with 5 to 8) -- is launch-bound, and its whole sync is ONE kernel: every
+ * thread block recomputes steps 1 and 2 from the K losses, and the block that
+ * draws the last ticket of a counter publishes g, the improved mask, pBest_loss
+ * and the counter (no block waits for another).  Otherwise, or with
  * PSOPS_SEPARATE_SELECT, a selection kernel runs first and the update kernel
- * behind it.  The results are identical bit for bit.
+ * behind it.  A swarm of 9 or more particles on few elements (up to 2^19, and
+ * few enough that one block column per 1024 elements would leave SMs idle) has
+ * its rows split into groups that run side by side; since row g is then read
+ * by blocks that do not write it, a third small kernel first copies it into the
+ * workspace (selection, snapshot, update).  The results are identical bit for
+ * bit in every form.
  * Cache policy: of the arrays x, v, pbest (4 K N bytes each) as many as fit
  * together in about half of the GPU's L2 cache are accessed with ordinary
  * loads and stores, so that the next sync finds them there; the others, and

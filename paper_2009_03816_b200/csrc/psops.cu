@@ -90,6 +90,21 @@ bool config_ok(const psops_config *c)
 inline int swarm_size(const psops_config *c) { return c->K_total ? c->K_total : c->K; }
 inline bool keeps_gbest(const psops_config *c) { return (c->flags & (PSOPS_KEEP_GBEST | PSOPS_GBEST_HISTORY)) != 0; }
 
+// Many particles on few elements: the update splits the rows over blockIdx.y
+// (see psops_sync) and then needs a snapshot of the gBest row, N floats of
+// workspace.  Whether a swarm may be split depends on its shape only, so that
+// the workspace size does not depend on the device.
+#ifndef PSOPS_SPLIT_MAX_ELEMENTS
+#define PSOPS_SPLIT_MAX_ELEMENTS (1ll << 19)
+#endif
+constexpr int kSplitMinParticles = 9;           // below: the single-launch form or one group
+constexpr int kSplitRowsPerGroup = 4;           // at least this many rows per group (one full batch)
+inline bool may_split_rows(const psops_config *c)
+{
+    return c->K >= kSplitMinParticles && c->N <= PSOPS_SPLIT_MAX_ELEMENTS &&
+           !(c->flags & (PSOPS_QUADRATIC | PSOPS_GBEST_HISTORY)) && swarm_size(c) == c->K;
+}
+
 Layout make_layout(const psops_config *c)
 {
     Layout L{};
@@ -99,7 +114,7 @@ Layout make_layout(const psops_config *c)
     L.off_pbest_loss = at;  at += kbytes;
     L.off_desc = at;        at += round_up(sizeof(SyncDesc), 256);
     L.off_gbest = at;
-    if (keeps_gbest(c)) at += round_up(sizeof(float) * (size_t)round_up((size_t)c->N, 4), 256);
+    if (keeps_gbest(c) || may_split_rows(c)) at += round_up(sizeof(float) * (size_t)round_up((size_t)c->N, 4), 256);
     L.off_partials = at;
     if (c->flags & PSOPS_QUADRATIC) {
         const size_t tiles = ((size_t)c->N + kTileElems - 1) / kTileElems;
@@ -143,6 +158,9 @@ struct psops_ctx {
     int *d_g;                          // the same word as the device sees it
     cudaEvent_t ev_select;             // recorded behind the selection kernel of a shard
     int resident_arrays;               // how many of x, v, pbest are accessed write-back (kept in L2); the rest is streamed
+    float *d_snapshot;                 // N floats for the gBest snapshot of a row-split update (the kept copy, if one is kept)
+    int row_groups;                    // > 1: psops_sync splits the rows into this many groups over blockIdx.y
+    int group_rows;                    // rows per group
     long long one_wave_blocks;         // blocks of the select-in-update kernel that are resident at once on this GPU
     int Kt;                            // particles in the whole swarm (= cfg.K unless sharded)
     uint32_t step;                     // syncs enqueued through this context (the stream's own counter is on the device)
@@ -261,9 +279,10 @@ constexpr int kUnrollFew = 1;
 // is as deep as the swarm: four particles in flight up to K = 4, eight beyond
 // (152 registers, one block per SM, hence a smaller "one wave").  Measured per
 // sync from a CUDA graph, N = 61,706: K = 4: 4.4 us; K = 8: 6.8 us (7.9 with
-// four in flight, 7.6 as two kernels); K = 16: 12.3 (13.7 / 12.2); K = 32 is
-// faster as two kernels (21 vs 23 us) and keeps them.
-constexpr int kSelectMaxParticles = 16;
+// four in flight, 7.6 as two kernels).  More particles than that on few
+// elements are better served by splitting the rows over more blocks (see
+// psops_sync).
+constexpr int kSelectMaxParticles = 8;
 constexpr int kUnrollSelectDeep = 8;
 static_assert(32 % kUnrollSelectDeep == 0 && kSelectMaxParticles <= 32, "one improved-mask word, reloaded every 32 particles");
 
@@ -302,7 +321,7 @@ UpdateKernel pick_update_kernel(bool aligned, bool fitness, bool select, int res
 // also does the selection of this sync (whole range, K <= 32, see the kernel).
 int launch_update(psops_ctx *ctx, float m, float k1, float k2, long long q_begin,
                   long long q_end, bool fitness, cudaStream_t stream, bool programmatic = false,
-                  bool select = false, const float *gbest_ext = nullptr)
+                  bool select = false, const float *gbest_ext = nullptr, bool split_rows = false)
 {
     if (q_end <= q_begin) return PSOPS_OK;
     UpdateParams P{};
@@ -318,15 +337,18 @@ int launch_update(psops_ctx *ctx, float m, float k1, float k2, long long q_begin
     P.q_begin = q_begin; P.q_end = q_end;
     P.tiles = ctx->tiles;
     P.K = ctx->cfg.K;
+    P.group_rows = split_rows ? ctx->group_rows : ctx->cfg.K;
+    if (split_rows) P.gbest_copy = nullptr;         // gbest_ext is the snapshot, which is also the kept copy
     P.m = m; P.k1 = k1; P.k2 = k2;
     fill_round_keys(ctx->cfg.seed, P.rk);
     const long long span = q_end - q_begin;
     const int per_block = kUpdateThreads * (fitness ? kFitQuads : kQuads);
     const unsigned blocks = (unsigned)((span + per_block - 1) / per_block);
     const bool few = ctx->cfg.K <= kFewParticles && (long long)blocks > ctx->one_wave_blocks;
+    const unsigned groups = split_rows ? (unsigned)ctx->row_groups : 1u;
     const UpdateKernel kernel = pick_update_kernel(ctx->aligned, fitness, select, ctx->resident_arrays, few, ctx->cfg.K);
     if (kernel == nullptr) return PSOPS_EINVAL;
-    const cudaError_t e = launch_serialized(programmatic, kernel, dim3(blocks, 1, 1), dim3(kUpdateThreads, 1, 1), stream, P);
+    const cudaError_t e = launch_serialized(programmatic, kernel, dim3(blocks, groups, 1), dim3(kUpdateThreads, 1, 1), stream, P);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "psops_update_kernel launch");
     if (select) ctx->loss_src = ctx->d_losses;      // the launch keeps a copy there
     return check_launch(ctx, "psops_update_kernel");
@@ -428,6 +450,9 @@ int psops_create(psops_ctx **out, const psops_config *cfg, float *d_x, float *d_
     ctx->d_pbest_loss = (float *)(ctx->ws + lay.off_pbest_loss);
     ctx->d_desc = (SyncDesc *)(ctx->ws + lay.off_desc);
     ctx->d_gbest = keeps_gbest(cfg) ? (float *)(ctx->ws + lay.off_gbest) : nullptr;
+    ctx->d_snapshot = (keeps_gbest(cfg) || may_split_rows(cfg)) ? (float *)(ctx->ws + lay.off_gbest) : nullptr;
+    ctx->row_groups = 1;
+    ctx->group_rows = cfg->K;
     ctx->Kt = swarm_size(cfg);
     ctx->selected = false;
     ctx->range_next = 0;
@@ -475,6 +500,23 @@ int psops_create(psops_ctx **out, const psops_config *cfg, float *d_x, float *d_
                 &per_sm, pick_update_kernel(ctx->aligned, false, true, ctx->resident_arrays, false, cfg->K),
                 kUpdateThreads, 0);
         ctx->one_wave_blocks = (long long)sms * per_sm;
+        // Rows split into groups when one group per column block would leave most
+        // of the GPU idle: as many groups as fit in one wave of the plain kernel,
+        // each with at least one full batch of rows.
+        if (e == cudaSuccess && may_split_rows(cfg)) {
+            int plain_per_sm = 0;
+            e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+                &plain_per_sm, pick_update_kernel(ctx->aligned, false, false, ctx->resident_arrays, false, cfg->K),
+                kUpdateThreads, 0);
+            const long long column_blocks = (ctx->quads + (long long)kUpdateThreads * kQuads - 1) / ((long long)kUpdateThreads * kQuads);
+            long long groups = (long long)sms * plain_per_sm / column_blocks;
+            const long long most = (cfg->K + kSplitRowsPerGroup - 1) / kSplitRowsPerGroup;
+            if (groups > most) groups = most;
+            if (e == cudaSuccess && groups >= 2) {
+                ctx->group_rows = (int)((cfg->K + groups - 1) / groups);
+                ctx->row_groups = (cfg->K + ctx->group_rows - 1) / ctx->group_rows;
+            }
+        }
     }
     if (e == cudaSuccess) {
         // pBest_loss <- +inf (Algorithm 2 clones weights only), descriptor <- 0.
@@ -525,7 +567,7 @@ int psops_sync(psops_ctx *ctx, int64_t t_iter, float lambda)
     const float k2 = ctx->cfg.c2 / lambda;
     const bool fitness = ctx->dvec != nullptr;
 
-    // A small swarm (at most 16 particles, all blocks of the update resident at
+    // A small swarm (at most 8 particles, all blocks of the update resident at
     // once) is launch-bound: there the update launch does the selection itself,
     // one kernel per sync.  Anything larger, the history variant and the fused
     // fitness run the selection kernel first and the update behind it, which
@@ -538,10 +580,30 @@ int psops_sync(psops_ctx *ctx, int64_t t_iter, float lambda)
         rc = launch_select(ctx);
         if (rc != PSOPS_OK) return rc;
     }
+    // Many particles on few elements: one thread walking all K rows would leave
+    // most SMs idle, so the rows are split into groups over blockIdx.y.  Row g
+    // is then read by blocks that do not write it: it is copied to a snapshot
+    // first (selection -> snapshot -> update, each launched programmatically
+    // behind the other).
+    const bool split_rows = ctx->row_groups > 1 && !fitness && !select_in_update;
+    if (split_rows) {
+        const unsigned blocks = (unsigned)((ctx->quads + kUpdateThreads - 1) / kUpdateThreads);
+        const cudaError_t e = ctx->aligned
+            ? launch_serialized(true, psops_gbest_snapshot_kernel<true>, dim3(blocks, 1, 1), dim3(kUpdateThreads, 1, 1),
+                                ctx->stream, (const SyncDesc *)ctx->d_desc, (const float *)ctx->x,
+                                (long long)ctx->cfg.ld, (long long)ctx->cfg.N, ctx->quads, ctx->d_snapshot)
+            : launch_serialized(true, psops_gbest_snapshot_kernel<false>, dim3(blocks, 1, 1), dim3(kUpdateThreads, 1, 1),
+                                ctx->stream, (const SyncDesc *)ctx->d_desc, (const float *)ctx->x,
+                                (long long)ctx->cfg.ld, (long long)ctx->cfg.N, ctx->quads, ctx->d_snapshot);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "psops_gbest_snapshot_kernel launch");
+        rc = check_launch(ctx, "psops_gbest_snapshot_kernel");
+        if (rc != PSOPS_OK) return rc;
+    }
     // With the fused fitness every warp of a tile must be whole: round the
     // quad range up to a tile; quads past the end contribute +0.0.
     const long long q_end = fitness ? ctx->tiles * 32 : ctx->quads;
-    rc = launch_update(ctx, m, k1, k2, 0, q_end, fitness, ctx->stream, /*programmatic=*/true, select_in_update);
+    rc = launch_update(ctx, m, k1, k2, 0, q_end, fitness, ctx->stream, /*programmatic=*/true, select_in_update,
+                       split_rows ? ctx->d_snapshot : nullptr, split_rows);
     if (rc != PSOPS_OK) return rc;
     if (fitness) {
         rc = launch_finalize(ctx);

@@ -50,6 +50,7 @@ struct UpdateParams {
     long long q_begin, q_end;   // quad range of this launch (quad = 4 elements)
     long long tiles;            // ceil(N / 128)
     int K;                      // rows held here
+    int group_rows;             // rows one block works on: K, or less when blockIdx.y splits the rows into groups
     int i_first;                // swarm-wide index of row 0 (0 unless the swarm is sharded by particle)
     float m, k1, k2;            // inertia, c1/lambda, c2/lambda
     uint32_t rk[20];            // Philox round keys, rk[2r], rk[2r+1]
@@ -341,7 +342,7 @@ psops_select_kernel(const float *loss, float *loss_keep, float *__restrict__ pbe
 // contiguous piece of each row, which is what DRAM and the TLB like when K
 // rows x 3 arrays are all being walked at once.
 //
-// SELECT (K <= 32 by construction, used up to 16; whole-range launches only): the launch does the selection
+// SELECT (K <= 32 by construction, used up to 8; whole-range launches only): the launch does the selection
 // as well, so that a sync is ONE kernel.  Every warp recomputes Algorithm 3
 // and the pBest comparisons from the K losses (K L2-served floats and a
 // five-stage shuffle) and then draws a ticket from an atomic counter.  The
@@ -390,6 +391,16 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
         col[j] = (size_t)d0;
     }
     const int lane = threadIdx.x & 31;
+
+    // Rows this block works on: all K of them, or -- for a swarm of many
+    // particles and few elements, which would otherwise leave most SMs idle
+    // while each thread walks all K rows -- the group blockIdx.y picks.  A
+    // launch that splits the rows is always given gBest in a buffer of its own
+    // (P.gbest_ext): the block that overwrites row g is then no longer the only
+    // one that reads it.
+    const int k0 = (int)blockIdx.y * P.group_rows;
+    const int Kg = (P.K - k0 < P.group_rows) ? P.K - k0 : P.group_rows;
+    const int ifirst = P.i_first + k0;       // swarm-wide index of this block's first row
 
     // Selection results: read from the descriptor the selection kernel filled,
     // or (SELECT) recomputed here by every warp; lane i stands for particle i.
@@ -461,19 +472,19 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
         for (int j = 0; j < Q; ++j) {
             fitness_tile_sums<U>(fq[j], lane);
             const int i = fq_i0 + fitness_row_of_lane<U>(lane);
-            if (fitness_lane_writes<U>(lane) && active[j] && i < P.K)   // q_end is a whole number of tiles
-                P.partials[(size_t)i * (size_t)P.tiles + (col[j] >> 7)] = fq[j][0];
+            if (fitness_lane_writes<U>(lane) && active[j] && i < Kg)    // q_end is a whole number of tiles
+                P.partials[(size_t)(k0 + i) * (size_t)P.tiles + (col[j] >> 7)] = fq[j][0];
         }
     };
 
-    size_t row = 0;                          // offset of row i0
-    uint32_t impw = sel_word;                // improved bits of particles i0 - i0 % 32 .. +31 (local numbering)
-    for (int i0 = 0; i0 < P.K; i0 += U) {
+    size_t row = (size_t)k0 * (size_t)P.ld;  // offset of row i0 of this block's group
+    uint32_t impw = sel_word;                // improved bits of particles i0 - i0 % 32 .. +31 (the group's numbering)
+    for (int i0 = 0; i0 < Kg; i0 += U) {
         if (!SELECT && (i0 & 31) == 0) {
             // One window of 32 bits per 32 particles, fetched ahead of the loads it
             // steers: a per-particle fetch would sit between them and stall the
             // in-order issue.  The window starts at swarm-wide particle i_first + i0.
-            const int base = P.i_first + i0;
+            const int base = ifirst + i0;
             const uint32_t lo = P.desc->improved[base >> 5];
             const uint32_t hi = ((base >> 5) + 1 < PSOPS_MAX_K / 32) ? P.desc->improved[(base >> 5) + 1] : 0u;
             impw = __funnelshift_r(lo, hi, base & 31);
@@ -485,7 +496,7 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
         for (int u = 0; u < U; ++u) {
             const int i = i0 + u;
             imp[u] = (impw >> (i & 31)) & 1u;
-            if (i < P.K) {
+            if (i < Kg) {
 #pragma unroll
                 for (int j = 0; j < Q; ++j) {
                     const size_t at = row + (size_t)u * (size_t)P.ld + col[j];
@@ -528,14 +539,14 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int i = i0 + u;
-            if (i < P.K) {
+            if (i < Kg) {
 #pragma unroll
                 for (int j = 0; j < Q; ++j) {
                     const size_t at = row + (size_t)u * (size_t)P.ld + col[j];
                     const uint32_t pair = pair0 + (uint32_t)(2 * j * kUpdateThreads);
                     uint32_t ra[4], rb[4];
-                    philox4x32_10(pair, (uint32_t)(P.i_first + i), step, 0u, P.rk, ra);
-                    philox4x32_10(pair + 1u, (uint32_t)(P.i_first + i), step, 0u, P.rk, rb);
+                    philox4x32_10(pair, (uint32_t)(ifirst + i), step, 0u, P.rk, ra);
+                    philox4x32_10(pair + 1u, (uint32_t)(ifirst + i), step, 0u, P.rk, rb);
                     const uint32_t w1[4] = {ra[0], ra[2], rb[0], rb[2]};   // r1 of elements 0..3
                     const uint32_t w2[4] = {ra[1], ra[3], rb[1], rb[3]};   // r2 of elements 0..3
                     float vn[4], xn[4];
@@ -562,6 +573,27 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
     }
     if (FITNESS && fq_i0 >= 0) flush_fitness();
 
+}
+
+// ---------------------------------------------------------------------------
+// gBest snapshot for launches of kernel (b) that split the rows over
+// blockIdx.y: row g of x, as the selection kernel in front of it chose it, is
+// copied to `dst` before the update overwrites it.
+// ---------------------------------------------------------------------------
+template <bool ALIGNED>
+__global__ void __launch_bounds__(kUpdateThreads)
+psops_gbest_snapshot_kernel(const SyncDesc *__restrict__ desc, const float *__restrict__ x, long long ld,
+                            long long N, long long quads, float *__restrict__ dst)
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");         // the selection kernel has written desc->g
+    const long long q = (long long)blockIdx.x * kUpdateThreads + threadIdx.x;
+    if (q >= quads) return;
+    const long long d0 = q * 4;
+    const int nvalid = (N - d0 >= 4) ? 4 : (int)(N - d0);
+    float a[4];
+    load_quad_cached<ALIGNED>(x + (size_t)desc->g * (size_t)ld + d0, nvalid, a);
+    store_quad<ALIGNED, false>(dst + d0, nvalid, a);
 }
 
 // ---------------------------------------------------------------------------

@@ -34,10 +34,11 @@ def _swarm(K, N, seed, sv=0.1):
 @pytest.mark.parametrize("K,separate", [(1, False), (2, False), (3, False), (5, False), (8, False), (16, False),
                                         (1, True), (2, True), (3, True), (8, True), (32, True), (33, True)])
 def test_small_shapes_vector_path(K, N, separate):
-    """Up to 16 particles a small sync is one launch that selects and updates
-    (four particles in flight up to K = 4, eight beyond);
-    PSOPS_SEPARATE_SELECT (and any larger swarm) runs the selection kernel
-    first.  Both must follow the oracle bit for bit."""
+    """Up to 8 particles a small sync is one launch that selects and updates
+    (four particles in flight up to K = 4, eight beyond); PSOPS_SEPARATE_SELECT
+    runs the selection kernel first; 9 or more particles on so few elements
+    have their rows split over more blocks (selection, gBest snapshot,
+    update).  All must follow the oracle bit for bit."""
     x, v, p = _swarm(K, N, 100 * K + N)
     pair = Pair(x, v, p, N, m_max=0.9, m_min=0.3, t_max=10, c1=0.2, c2=0.9, seed=K * 7919 + N,
                 flags=PSOPS_SEPARATE_SELECT if separate else 0)
@@ -48,7 +49,7 @@ def test_small_shapes_vector_path(K, N, separate):
         pair.check_state(f"K={K} N={N} s={s}")
     pair.check_canaries()
     assert pair.inexact == 0          # same rounding sequence on both sides
-    assert pair.gpu.launches == (8 if separate else 4)
+    assert pair.gpu.launches == (12 if K >= 9 else 8 if separate else 4)
     pair.close()
 
 
@@ -85,7 +86,7 @@ def test_many_particles():
 # ---------------------------------------------------------------------------
 # Selection edge cases through the device kernel.
 # ---------------------------------------------------------------------------
-@pytest.mark.parametrize("K", [7, 12, 16, 20, 40])    # selection inside the update launch (K <= 16) / selection kernel
+@pytest.mark.parametrize("K", [7, 8, 12, 20, 40])     # selection inside the update launch (K <= 8) / selection kernel
 def test_selection_ties_nan_inf_on_device(K):
     N = 64
     x, v, p = _swarm(K, N, 9)
@@ -119,9 +120,11 @@ def test_selection_ties_nan_inf_on_device(K):
     pair.close()
 
 
+@pytest.mark.parametrize("K", [5, 13])                 # 13: rows split into groups, gBest read from a snapshot
 @pytest.mark.parametrize("g", [0, 1, 2, 3, 4])
-def test_gbest_row_is_read_before_it_is_overwritten(g):
-    K, N = 5, 10_007
+def test_gbest_row_is_read_before_it_is_overwritten(g, K):
+    N = 10_007
+    g = g if K == 5 else 3 * g                           # 0, 3, 6, 9, 12: a row of every group
     x, v, p = _swarm(K, N, 77)
     pair = Pair(x, v, p, N, m_max=0.7, m_min=0.7, c1=1.5, c2=1.5, seed=g, flags=PSOPS_KEEP_GBEST)
     loss = np.full(K, 2.0, np.float32)
