@@ -289,7 +289,7 @@ static_assert(32 % kUnrollSelectDeep == 0 && kSelectMaxParticles <= 32, "one imp
 // All instantiations of kernel (b) for one alignment and one cache policy
 // (`resident` arrays of x, v, pbest accessed write-back, the rest streamed).
 struct UpdateKernelSet {
-    UpdateKernel plain, select, select_deep, few, fitness;
+    UpdateKernel plain, select, select_deep, few, fitness, split;
 };
 
 template <bool ALIGNED, int RESIDENT>
@@ -299,10 +299,12 @@ constexpr UpdateKernelSet update_kernel_set()
             psops_update_kernel<ALIGNED, false, true, RESIDENT, kUnroll, kQuads>,
             psops_update_kernel<ALIGNED, false, true, RESIDENT, kUnrollSelectDeep, kQuads>,
             psops_update_kernel<ALIGNED, false, false, RESIDENT, kUnrollFew, kQuads>,
-            psops_update_kernel<ALIGNED, true, false, RESIDENT, kFitUnroll, kFitQuads>};
+            psops_update_kernel<ALIGNED, true, false, RESIDENT, kFitUnroll, kFitQuads>,
+            psops_update_kernel<ALIGNED, false, false, RESIDENT, kUnroll, kQuads, true>};
 }
 
-UpdateKernel pick_update_kernel(bool aligned, bool fitness, bool select, int resident, bool few, int K)
+UpdateKernel pick_update_kernel(bool aligned, bool fitness, bool select, int resident, bool few, int K,
+                                bool split = false)
 {
     static const UpdateKernelSet sets[2][4] = {
         {update_kernel_set<false, 0>(), update_kernel_set<false, 1>(), update_kernel_set<false, 2>(),
@@ -312,6 +314,7 @@ UpdateKernel pick_update_kernel(bool aligned, bool fitness, bool select, int res
     };
     if (resident < 0 || resident > 3 || (fitness && select)) return nullptr;
     const UpdateKernelSet &set = sets[aligned ? 1 : 0][resident];
+    if (split) return (fitness || select) ? nullptr : set.split;
     if (fitness) return set.fitness;
     if (select) return K > kUnroll ? set.select_deep : set.select;
     return few ? set.few : set.plain;
@@ -346,7 +349,8 @@ int launch_update(psops_ctx *ctx, float m, float k1, float k2, long long q_begin
     const unsigned blocks = (unsigned)((span + per_block - 1) / per_block);
     const bool few = ctx->cfg.K <= kFewParticles && (long long)blocks > ctx->one_wave_blocks;
     const unsigned groups = split_rows ? (unsigned)ctx->row_groups : 1u;
-    const UpdateKernel kernel = pick_update_kernel(ctx->aligned, fitness, select, ctx->resident_arrays, few, ctx->cfg.K);
+    const UpdateKernel kernel = pick_update_kernel(ctx->aligned, fitness, select, ctx->resident_arrays, few, ctx->cfg.K,
+                                                   split_rows);
     if (kernel == nullptr) return PSOPS_EINVAL;
     const cudaError_t e = launch_serialized(programmatic, kernel, dim3(blocks, groups, 1), dim3(kUpdateThreads, 1, 1), stream, P);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "psops_update_kernel launch");
@@ -506,7 +510,7 @@ int psops_create(psops_ctx **out, const psops_config *cfg, float *d_x, float *d_
         if (e == cudaSuccess && may_split_rows(cfg)) {
             int plain_per_sm = 0;
             e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-                &plain_per_sm, pick_update_kernel(ctx->aligned, false, false, ctx->resident_arrays, false, cfg->K),
+                &plain_per_sm, pick_update_kernel(ctx->aligned, false, false, ctx->resident_arrays, false, cfg->K, true),
                 kUpdateThreads, 0);
             const long long column_blocks = (ctx->quads + (long long)kUpdateThreads * kQuads - 1) / ((long long)kUpdateThreads * kQuads);
             long long groups = (long long)sms * plain_per_sm / column_blocks;

@@ -74,13 +74,18 @@ struct UpdateParams {
 #define PSOPS_FITNESS_QUADS 1
 #endif
 #ifndef PSOPS_UPDATE_MIN_BLOCKS
-#define PSOPS_UPDATE_MIN_BLOCKS 0      // >0: resident blocks per SM the register allocation must allow
+#define PSOPS_UPDATE_MIN_BLOCKS 0      // >0: resident blocks per SM the register allocation must allow (0: compiler's choice)
 #endif
-#if PSOPS_UPDATE_MIN_BLOCKS > 0
-#define PSOPS_UPDATE_BOUNDS __launch_bounds__(PSOPS_UPDATE_THREADS, PSOPS_UPDATE_MIN_BLOCKS)
-#else
-#define PSOPS_UPDATE_BOUNDS __launch_bounds__(PSOPS_UPDATE_THREADS)
+#ifndef PSOPS_FITNESS_MIN_BLOCKS
+#define PSOPS_FITNESS_MIN_BLOCKS 4     // the same with the fitness fused in: 64 registers, four blocks of 256 threads
 #endif
+// Left to itself the compiler gives the streaming variants 80 registers (three
+// blocks per SM), which is what they were tuned at; the all-resident plain
+// variant it would take to 105, so that one is held at three blocks as well.
+#define PSOPS_UPDATE_BOUNDS                                                          \
+    __launch_bounds__(PSOPS_UPDATE_THREADS,                                          \
+                      (FITNESS ? PSOPS_FITNESS_MIN_BLOCKS                            \
+                               : (!SELECT && RESIDENT == 3 && U > 1) ? 3 : PSOPS_UPDATE_MIN_BLOCKS))
 constexpr int kUpdateThreads = PSOPS_UPDATE_THREADS;
 constexpr int kFinalizeThreads = 1024;     // = number of level-2 slots
 constexpr int kTileElems = 128;            // one warp x one quad per lane
@@ -359,7 +364,7 @@ psops_select_kernel(const float *loss, float *loss_keep, float *__restrict__ pbe
 // ones, which the next sync finds there (x and v are read AND written each
 // sync, pbest only one of the two, hence the order).
 // ---------------------------------------------------------------------------
-template <bool ALIGNED, bool FITNESS, bool SELECT, int RESIDENT, int U, int Q>
+template <bool ALIGNED, bool FITNESS, bool SELECT, int RESIDENT, int U, int Q, bool SPLIT = false>
 __global__ void PSOPS_UPDATE_BOUNDS
 psops_update_kernel(const __grid_constant__ UpdateParams P)
 {
@@ -398,8 +403,9 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
     // launch that splits the rows is always given gBest in a buffer of its own
     // (P.gbest_ext): the block that overwrites row g is then no longer the only
     // one that reads it.
-    const int k0 = (int)blockIdx.y * P.group_rows;
-    const int Kg = (P.K - k0 < P.group_rows) ? P.K - k0 : P.group_rows;
+    // (SPLIT is a compile-time switch so that the ordinary launches carry none of it.)
+    const int k0 = SPLIT ? (int)blockIdx.y * P.group_rows : 0;
+    const int Kg = SPLIT ? ((P.K - k0 < P.group_rows) ? P.K - k0 : P.group_rows) : P.K;
     const int ifirst = P.i_first + k0;       // swarm-wide index of this block's first row
 
     // Selection results: read from the descriptor the selection kernel filled,
