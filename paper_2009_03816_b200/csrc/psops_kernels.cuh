@@ -50,10 +50,11 @@ struct UpdateParams {
     long long q_begin, q_end;   // quad range of this launch (quad = 4 elements)
     long long tiles;            // ceil(N / 128)
     int K;                      // rows held here
-    int group_rows;             // rows one block works on: K, or less when blockIdx.y splits the rows into groups
     int i_first;                // swarm-wide index of row 0 (0 unless the swarm is sharded by particle)
     float m, k1, k2;            // inertia, c1/lambda, c2/lambda
     uint32_t rk[20];            // Philox round keys, rk[2r], rk[2r+1]
+    int group_rows;             // rows one block works on: K, or less when blockIdx.y splits the rows into groups
+                                // (last on purpose: the members above keep the offsets the kernels were tuned with)
 };
 
 // Launch shape of the streaming kernels; the defaults are the measured best on
@@ -403,10 +404,13 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
     // launch that splits the rows is always given gBest in a buffer of its own
     // (P.gbest_ext): the block that overwrites row g is then no longer the only
     // one that reads it.
-    // (SPLIT is a compile-time switch so that the ordinary launches carry none of it.)
+    // SPLIT is a compile-time switch so that the ordinary launches carry none of
+    // it: their row count is written as the kernel parameter itself below (a
+    // local copy of it cost the one-particle-in-flight variant 15 %).
     const int k0 = SPLIT ? (int)blockIdx.y * P.group_rows : 0;
-    const int Kg = SPLIT ? ((P.K - k0 < P.group_rows) ? P.K - k0 : P.group_rows) : P.K;
+    const int Kg = (P.K - k0 < P.group_rows) ? P.K - k0 : P.group_rows;   // used with SPLIT only
     const int ifirst = P.i_first + k0;       // swarm-wide index of this block's first row
+#define PSOPS_ROWS (SPLIT ? Kg : P.K)
 
     // Selection results: read from the descriptor the selection kernel filled,
     // or (SELECT) recomputed here by every warp; lane i stands for particle i.
@@ -478,14 +482,14 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
         for (int j = 0; j < Q; ++j) {
             fitness_tile_sums<U>(fq[j], lane);
             const int i = fq_i0 + fitness_row_of_lane<U>(lane);
-            if (fitness_lane_writes<U>(lane) && active[j] && i < Kg)    // q_end is a whole number of tiles
+            if (fitness_lane_writes<U>(lane) && active[j] && i < PSOPS_ROWS)    // q_end is a whole number of tiles
                 P.partials[(size_t)(k0 + i) * (size_t)P.tiles + (col[j] >> 7)] = fq[j][0];
         }
     };
 
     size_t row = (size_t)k0 * (size_t)P.ld;  // offset of row i0 of this block's group
     uint32_t impw = sel_word;                // improved bits of particles i0 - i0 % 32 .. +31 (the group's numbering)
-    for (int i0 = 0; i0 < Kg; i0 += U) {
+    for (int i0 = 0; i0 < PSOPS_ROWS; i0 += U) {
         if (!SELECT && (i0 & 31) == 0) {
             // One window of 32 bits per 32 particles, fetched ahead of the loads it
             // steers: a per-particle fetch would sit between them and stall the
@@ -502,7 +506,7 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
         for (int u = 0; u < U; ++u) {
             const int i = i0 + u;
             imp[u] = (impw >> (i & 31)) & 1u;
-            if (i < Kg) {
+            if (i < PSOPS_ROWS) {
 #pragma unroll
                 for (int j = 0; j < Q; ++j) {
                     const size_t at = row + (size_t)u * (size_t)P.ld + col[j];
@@ -545,7 +549,7 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int i = i0 + u;
-            if (i < Kg) {
+            if (i < PSOPS_ROWS) {
 #pragma unroll
                 for (int j = 0; j < Q; ++j) {
                     const size_t at = row + (size_t)u * (size_t)P.ld + col[j];
@@ -578,7 +582,7 @@ psops_update_kernel(const __grid_constant__ UpdateParams P)
         row += (size_t)U * (size_t)P.ld;
     }
     if (FITNESS && fq_i0 >= 0) flush_fitness();
-
+#undef PSOPS_ROWS
 }
 
 // ---------------------------------------------------------------------------
