@@ -42,8 +42,8 @@ FALLBACK_HBM_GBS = 6650.0           # earlier measurement on this machine, used onl
 # source it was taken from: everything in psops_kernels.cuh up to the averaging
 # kernel, i.e. the update kernel and all it uses.  The benchmark reports null
 # once that text has changed, and for workloads whose state is kept in L2.
-NCU_TRAFFIC = {"source_sha256": "d448d23e432aa7864fd7fa18d83d6a1448395e41748935489e7be709c6df83fc",
-               "bytes_per_particle_element": 19.56,       # 2.506 / 2.503 GB per launch over 128 M: cfg4 recipe at N = 4 M
+NCU_TRAFFIC = {"source_sha256": "3f17bcc27ebf804f3d54929b581d77907043aafa69e805acbc4ed6d7fe14f1f6",
+               "bytes_per_particle_element": 19.56,       # 2.505 / 2.503 GB per launch over 128 M: cfg4 recipe at N = 4 M
                "profile": "profiles/update_kernel_cfg4_n4m.txt"}
 KERNEL_SOURCE = os.path.join(ROOT, "paper_2009_03816_b200", "csrc", "psops_kernels.cuh")
 HASH_UNTIL = "// Kernel (c): parameter averaging"
