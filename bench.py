@@ -735,8 +735,12 @@ def other_rows(args, dev, ranks, peak):
         sw.close()
         del sw, keep
         torch.cuda.empty_cache()
-        for name in (() if args.n else ("cfg1", "cfg2")):
-            ws = workloads.CONFIGS[name]
+        # small swarms: cfg1, cfg2, and the paper's own regime of many workers on a LeNet-sized vector
+        # (the cfg3 / cfg4 recipes with 16 / 32 particles at cfg1's 61,706 elements)
+        small = {"cfg1": workloads.CONFIGS["cfg1"], "cfg2": workloads.CONFIGS["cfg2"],
+                 "k16_n61706": workloads.CONFIGS["cfg3"].scaled(N=61_706),
+                 "k32_n61706": workloads.CONFIGS["cfg4"].scaled(N=61_706)}
+        for name, ws in (() if args.n else small.items()):
             cols = workloads.sample_columns_dense(ws.N, PARITY_COLUMNS, ws.seed) if check else None
             # no further windows here: cfg2's omega = 0.9, c = 2 lies outside PSO's stability region, and a
             # few hundred syncs beyond its 50 would overflow fp32 and leave nothing finite to compare
