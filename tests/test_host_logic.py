@@ -50,6 +50,16 @@ def test_workspace_bytes(lib):
     quad = binding.make_config(8, 1000, m_max=0.7, m_min=0.7, c1=1.5, c2=1.5, seed=1,
                                flags=binding.PSOPS_QUADRATIC)
     assert binding.psops_workspace_bytes(quad) >= n0 + 8 * 8 * 8      # K x ceil(N/128) doubles
+    # many particles on few elements: the update may split the rows over more blocks and then keeps
+    # a snapshot of the gBest row in the workspace -- by the swarm's shape alone, whatever the device
+    many = binding.make_config(16, 1000, m_max=0.7, m_min=0.7, c1=1.5, c2=1.5, seed=1)
+    few = binding.make_config(8, 1000, m_max=0.7, m_min=0.7, c1=1.5, c2=1.5, seed=1)
+    big = binding.make_config(16, (1 << 19) + 4, m_max=0.7, m_min=0.7, c1=1.5, c2=1.5, seed=1)
+    assert binding.psops_workspace_bytes(many) >= binding.psops_workspace_bytes(few) + 4000
+    assert binding.psops_workspace_bytes(big) == binding.psops_workspace_bytes(many) - 4096
+    many_kept = binding.make_config(16, 1000, m_max=0.7, m_min=0.7, c1=1.5, c2=1.5, seed=1,
+                                    flags=binding.PSOPS_KEEP_GBEST)
+    assert binding.psops_workspace_bytes(many_kept) == binding.psops_workspace_bytes(many)   # one row serves both
     for bad in (dict(K=0), dict(K=1025), dict(N=0), dict(N=1 << 33), dict(ld=999), dict(t_max=0),
                 dict(flags=16), dict(c1=float("nan")), dict(m_max=float("inf"))):
         kw = dict(K=8, N=1000, ld=1000, m_max=0.7, m_min=0.7, t_max=1, c1=1.5, c2=1.5, seed=1, flags=0)
