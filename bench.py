@@ -39,14 +39,14 @@ FALLBACK_HBM_GBS = 6650.0           # earlier measurement on this machine, used onl
 # DRAM traffic of the fused update kernel from an ncu capture of a small case
 # (N = 4 M, state larger than L2), per particle-element -- every value is
 # touched once, so traffic grows in proportion to K x N -- and the hash of the
-# source it was taken from: everything in psops_kernels.cuh up to the averaging
-# kernel, i.e. the update kernel and all it uses.  The benchmark reports null
+# source it was taken from: everything in psops_kernels.cuh up to the end of the
+# update kernel, i.e. that kernel and all it uses.  The benchmark reports null
 # once that text has changed, and for workloads whose state is kept in L2.
-NCU_TRAFFIC = {"source_sha256": "3f17bcc27ebf804f3d54929b581d77907043aafa69e805acbc4ed6d7fe14f1f6",
+NCU_TRAFFIC = {"source_sha256": "8a56c0c1a46a1f7c167811c1992ddba1753b9dd1379854339f3eecaa9faa6245",
                "bytes_per_particle_element": 19.56,       # 2.505 / 2.503 GB per launch over 128 M: cfg4 recipe at N = 4 M
                "profile": "profiles/update_kernel_cfg4_n4m.txt"}
 KERNEL_SOURCE = os.path.join(ROOT, "paper_2009_03816_b200", "csrc", "psops_kernels.cuh")
-HASH_UNTIL = "// Kernel (c): parameter averaging"
+HASH_UNTIL = "// gBest snapshot for launches of kernel (b)"
 
 
 def update_kernel_source_sha256() -> str:

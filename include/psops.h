@@ -147,9 +147,11 @@ int psops_set_losses(psops_ctx *ctx, const float *losses, int on_device);
  * behind it.  A swarm of 9 or more particles on few elements (up to 2^19, and
  * few enough that one block column per 1024 elements would leave SMs idle) has
  * its rows split into groups that run side by side; since row g is then read
- * by blocks that do not write it, a third small kernel first copies it into the
- * workspace (selection, snapshot, update).  The results are identical bit for
- * bit in every form.
+ * by blocks that do not write it, a small kernel first copies it into the
+ * workspace -- up to 32 particles that kernel also does the selection (two
+ * launches per sync), beyond 32 or with PSOPS_SEPARATE_SELECT the selection
+ * kernel runs in front of it (three).  The results are identical bit for bit in
+ * every form.
  * Cache policy: of the arrays x, v, pbest (4 K N bytes each) as many as fit
  * together in about half of the GPU's L2 cache are accessed with ordinary
  * loads and stores, so that the next sync finds them there; the others, and

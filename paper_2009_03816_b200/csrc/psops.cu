@@ -580,17 +580,34 @@ int psops_sync(psops_ctx *ctx, int64_t t_iter, float lambda)
     const bool select_in_update = ctx->cfg.K <= kSelectMaxParticles && !fitness &&
                                   update_blocks <= ctx->one_wave_blocks &&
                                   !(ctx->cfg.flags & (PSOPS_GBEST_HISTORY | PSOPS_SEPARATE_SELECT));
-    if (!select_in_update) {
-        rc = launch_select(ctx);
-        if (rc != PSOPS_OK) return rc;
-    }
     // Many particles on few elements: one thread walking all K rows would leave
     // most SMs idle, so the rows are split into groups over blockIdx.y.  Row g
     // is then read by blocks that do not write it: it is copied to a snapshot
-    // first (selection -> snapshot -> update, each launched programmatically
-    // behind the other).
+    // first, by a kernel that up to 32 particles also does the selection
+    // (snapshot -> update; beyond 32: selection -> snapshot -> update), each
+    // launched programmatically behind the other.
     const bool split_rows = ctx->row_groups > 1 && !fitness && !select_in_update;
-    if (split_rows) {
+    const bool select_in_snapshot = split_rows && ctx->cfg.K <= 32 && !(ctx->cfg.flags & PSOPS_SEPARATE_SELECT);
+    if (!select_in_update && !select_in_snapshot) {
+        rc = launch_select(ctx);
+        if (rc != PSOPS_OK) return rc;
+    }
+    if (select_in_snapshot) {
+        const unsigned blocks = (unsigned)((ctx->quads + kUpdateThreads - 1) / kUpdateThreads);
+        const cudaError_t e = ctx->aligned
+            ? launch_serialized(true, psops_select_snapshot_kernel<true>, dim3(blocks, 1, 1), dim3(kUpdateThreads, 1, 1),
+                                ctx->stream, ctx->loss_src, ctx->d_losses, ctx->d_pbest_loss, ctx->d_desc, ctx->cfg.K,
+                                (const float *)ctx->x, (long long)ctx->cfg.ld, (long long)ctx->cfg.N, ctx->quads,
+                                ctx->d_snapshot)
+            : launch_serialized(true, psops_select_snapshot_kernel<false>, dim3(blocks, 1, 1), dim3(kUpdateThreads, 1, 1),
+                                ctx->stream, ctx->loss_src, ctx->d_losses, ctx->d_pbest_loss, ctx->d_desc, ctx->cfg.K,
+                                (const float *)ctx->x, (long long)ctx->cfg.ld, (long long)ctx->cfg.N, ctx->quads,
+                                ctx->d_snapshot);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "psops_select_snapshot_kernel launch");
+        ctx->loss_src = ctx->d_losses;              // the kernel keeps a copy there
+        rc = check_launch(ctx, "psops_select_snapshot_kernel");
+        if (rc != PSOPS_OK) return rc;
+    } else if (split_rows) {
         const unsigned blocks = (unsigned)((ctx->quads + kUpdateThreads - 1) / kUpdateThreads);
         const cudaError_t e = ctx->aligned
             ? launch_serialized(true, psops_gbest_snapshot_kernel<true>, dim3(blocks, 1, 1), dim3(kUpdateThreads, 1, 1),

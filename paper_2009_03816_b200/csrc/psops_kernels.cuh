@@ -606,6 +606,59 @@ psops_gbest_snapshot_kernel(const SyncDesc *__restrict__ desc, const float *__re
     store_quad<ALIGNED, false>(dst + d0, nvalid, a);
 }
 
+// The same snapshot with the selection folded in (K <= 32): every warp
+// recomputes Algorithm 3 and the pBest comparisons as in the single-launch
+// form of kernel (b), each thread copies its quad of row g, and the block that
+// draws the last ticket publishes the selection for the update kernel behind
+// it.  One launch instead of two in front of a row-split update.
+template <bool ALIGNED>
+__global__ void __launch_bounds__(kUpdateThreads)
+psops_select_snapshot_kernel(const float *loss_src, float *loss_keep, float *pbest_loss, SyncDesc *desc, int K,
+                             const float *__restrict__ x, long long ld, long long N, long long quads,
+                             float *__restrict__ dst)
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int lane = threadIdx.x & 31;
+    const bool live = lane < K;
+    const float li = live ? __ldcg(loss_src + lane) : 0.0f;
+    const float pl = live ? __ldcg(pbest_loss + lane) : 0.0f;
+    const bool improved = live && (li < pl);                 // strict: an equal loss never replaces pBest
+    const uint32_t word = __ballot_sync(0xffffffffu, improved);
+    Candidate c;
+    c.loss = live ? li : __int_as_float(0x7fc00000);
+    c.idx = live ? lane : 0x7fffffff;
+    const int g = warp_best_candidate(c).idx;
+    const uint32_t step = __ldcg(&desc->next_step);
+    __syncthreads();                                         // all warps of the block hold the old state in registers
+
+    const long long q = (long long)blockIdx.x * kUpdateThreads + threadIdx.x;
+    const long long d0 = q * 4;
+    const int nvalid = (q < quads) ? ((N - d0 >= 4) ? 4 : (int)(N - d0)) : 0;
+    float a[4];
+    load_quad_cached<ALIGNED>(x + (size_t)g * (size_t)ld + d0, nvalid, a);
+    if (threadIdx.x < 32) {                                  // the ticket, under the load just issued
+        unsigned int ticket = 0;
+        if (lane == 0) ticket = atomicAdd(&desc->done, 1u);
+        ticket = __shfl_sync(0xffffffffu, ticket, 0);
+        if (ticket == gridDim.x - 1) {                       // every block has read the old state: move it on
+            if (live) {
+                loss_keep[lane] = li;
+                if (improved) pbest_loss[lane] = li;
+            }
+            if (lane == 0) {
+                desc->g = g;
+                desc->improved[0] = word;
+                desc->from_kept = 0;
+                desc->step = step;
+                desc->next_step = step + 1u;
+                desc->done = 0u;
+            }
+        }
+    }
+    store_quad<ALIGNED, false>(dst + d0, nvalid, a);
+}
+
 // ---------------------------------------------------------------------------
 // Kernel (c): parameter averaging (Section II-B, step 5).
 // ---------------------------------------------------------------------------

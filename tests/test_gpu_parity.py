@@ -32,13 +32,14 @@ def _swarm(K, N, seed, sv=0.1):
 # ---------------------------------------------------------------------------
 @pytest.mark.parametrize("N", [1, 2, 3, 5, 127, 128, 129, 1000, 4099])
 @pytest.mark.parametrize("K,separate", [(1, False), (2, False), (3, False), (5, False), (8, False), (16, False),
-                                        (1, True), (2, True), (3, True), (8, True), (32, True), (33, True)])
+                                        (32, False), (1, True), (2, True), (3, True), (8, True), (32, True),
+                                        (33, True)])
 def test_small_shapes_vector_path(K, N, separate):
     """Up to 8 particles a small sync is one launch that selects and updates
     (four particles in flight up to K = 4, eight beyond); PSOPS_SEPARATE_SELECT
     runs the selection kernel first; 9 or more particles on so few elements
-    have their rows split over more blocks (selection, gBest snapshot,
-    update).  All must follow the oracle bit for bit."""
+    have their rows split over more blocks (a gBest snapshot that up to
+    32 particles also selects, then the update).  All must follow the oracle bit for bit."""
     x, v, p = _swarm(K, N, 100 * K + N)
     pair = Pair(x, v, p, N, m_max=0.9, m_min=0.3, t_max=10, c1=0.2, c2=0.9, seed=K * 7919 + N,
                 flags=PSOPS_SEPARATE_SELECT if separate else 0)
@@ -49,7 +50,10 @@ def test_small_shapes_vector_path(K, N, separate):
         pair.check_state(f"K={K} N={N} s={s}")
     pair.check_canaries()
     assert pair.inexact == 0          # same rounding sequence on both sides
-    assert pair.gpu.launches == (12 if K >= 9 else 8 if separate else 4)
+    # per sync: 1 launch (single-launch form), 2 (selection kernel + update, or selecting snapshot + row-split
+    # update), 3 (selection, snapshot, row-split update)
+    per_sync = 3 if (K > 32 or (K >= 9 and separate)) else 2 if (K >= 9 or separate) else 1
+    assert pair.gpu.launches == 4 * per_sync
     pair.close()
 
 
