@@ -528,8 +528,9 @@ def test_deterministic_and_resumable():
     sc.close()
 
 
-def test_sync_recorded_in_a_cuda_graph_replays_with_a_running_step_counter():
-    w = workloads.CONFIGS["cfg1"].scaled(N=40_001, S=8)
+@pytest.mark.parametrize("K", [4, 7, 16, 40])          # single launch (two depths), selecting snapshot + row-split
+def test_sync_recorded_in_a_cuda_graph_replays_with_a_running_step_counter(K):   # update, selection + snapshot + update
+    w = workloads.CONFIGS["cfg1"].scaled(N=40_001, S=8).with_particles(K)
     x, v, p = workloads.state(w)
     table = workloads.losses(w)
     stream = torch.cuda.Stream()
