@@ -1,7 +1,8 @@
 """CPU oracle for the PSO-PS synchronisation stage (test infrastructure).
 
-Only tests, the smoke check and the benchmark's CPU-baseline leg may import
-this package.  It never imports the CUDA package and the CUDA package never
+Only tests, the smoke check and the benchmark (its CPU-baseline and reference
+legs, and the check of the state it timed, all outside any timed region) may
+import this package.  It never imports the CUDA package and the CUDA package never
 imports it.
 """
 from .psops_oracle import (  # noqa: F401
